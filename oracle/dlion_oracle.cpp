@@ -1,0 +1,219 @@
+// Distributed Lion -- CPU oracle.
+//
+// TEST INFRASTRUCTURE ONLY.  This file is the slow, plain statement of what one
+// Distributed-Lion optimizer step computes.  It exists so that the CUDA library
+// can be checked against it.  It shares no code, header, table or helper with
+// the CUDA path and must never be called from the product path.
+//
+// What it follows (arXiv 2404.00438):
+//   * worker side  -- Algorithm 1 "Worker-side", and the pair of equations in
+//                     Section 3.2 that define m_{i,t+1} and delta_{i,t};
+//   * server side  -- Algorithm 1 "Server-side", and the aggregate(S_t)
+//                     equation of Section 3.2 (Averaging / Majority Vote);
+//   * apply        -- x_{i,t+1} = x_{i,t} - eps (Delta_t + lambda x_{i,t}),
+//                     last equation of Section 3.2;
+//   * wire format  -- Section 3.2 "Communication Cost" and Table 1: delta_i is a
+//                     binary vector of d bits; Delta is binary (Majority Vote) or
+//                     an integer in {0..N} (Averaging).
+//
+// The method is exact arithmetic on given inputs, so the oracle is the
+// definition written out coordinate by coordinate.  The paper does not fix the
+// floating-point format, the evaluation order, sign(0) or the even-N tie; the
+// readings used here are:
+//   R1  all arithmetic in IEEE binary32, one rounding per operation, no fused
+//       multiply-add (build with -ffp-contract=off):
+//           c   = fl( fl(beta1*m) + fl((1-beta1)*g) )
+//           m'  = fl( fl(beta2*m) + fl((1-beta2)*g) )
+//           x'  = fl( x - fl( eps * fl( Delta + fl(lambda*x) ) ) )
+//       with (1-beta) itself computed once in binary32.  bf16 gradients are
+//       widened exactly (bits << 16).
+//   R2  sgn(v) = +1 if v >= 0 else -1.  Both zeros give +1; NaN gives -1.  The
+//       wire carries one bit per coordinate, so sign has to be two-valued.
+//   R3  the same rule decides an even-N tie: S = 0 gives Delta = +1.
+//   R4  "S_t in {0..N}" is read as the count P of +1 votes; S = 2P - N.
+//   R5  delta_{i,t} uses the OLD momentum m_{i,t} (both equations carry the
+//       subscript t on their right-hand sides).
+//   R6  Averaging: Delta = (float)(2P-N) / (float)N, IEEE division.
+//
+// Parity status: every function below is pinned by tests/test_oracle_pins.py
+// (special cases N=1, identical workers, beta=0, beta1=beta2, brute-force vote
+// sums, closed forms for x and m in double precision, the Phase-I contraction of
+// Theorem "Phase I", a hand-derived worked example under tests/golden/).  The
+// one thing those cannot pin is reading R1 itself (the rounding order): the
+// paper is silent on it -- "parity unpinned" for the last-bit rounding order
+// only; the double-precision pins bound it to within an ulp per operation.
+//
+// Layout (the same conventions the C-ABI of the CUDA library documents, restated
+// here independently): arenas are worker-major, g[N][d_pad], m[N][d_pad],
+// packed[N][d_pad/32]; bit b of word w is coordinate 32*w+b; bit 1 means +1.
+// A segment table {elem_offset, numel} names the coordinates that are real
+// parameters; everything else is padding: never read as a parameter, never
+// written, and its packed bits are 0.
+
+#include <cstddef>
+#include <cstdint>
+#include <cstring>
+
+extern "C" {
+
+struct dlion_oracle_segment {
+    uint64_t elem_offset;
+    uint64_t numel;
+};
+
+enum { DLION_ORACLE_MAJORITY = 0, DLION_ORACLE_AVERAGE = 1 };
+enum { DLION_ORACLE_GRAD_F32 = 0, DLION_ORACLE_GRAD_BF16 = 1 };
+
+}  // extern "C"
+
+namespace {
+
+inline float widen_bf16(uint16_t h) {
+    uint32_t u = static_cast<uint32_t>(h) << 16;
+    float f;
+    std::memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+inline float load_grad(const void* g, int gdtype, size_t idx) {
+    if (gdtype == DLION_ORACLE_GRAD_BF16) {
+        return widen_bf16(static_cast<const uint16_t*>(g)[idx]);
+    }
+    return static_cast<const float*>(g)[idx];
+}
+
+// R2: two-valued sign as a bit.
+inline uint32_t sign_bit(float v) { return (v >= 0.0f) ? 1u : 0u; }
+
+}  // namespace
+
+extern "C" {
+
+// Worker side of Algorithm 1 for all N workers (or for one worker when the
+// caller passes N = 1 and that worker's slices).
+//   g       [N][d_pad]  gradients g_{i,t}, f32 or bf16            (read)
+//   m       [N][d_pad]  momenta m_{i,t} -> m_{i,t+1}, f32         (in place)
+//   packed  [N][d_pad/32] delta_{i,t}, one bit per coordinate     (written:
+//           words that hold at least one parameter; others untouched)
+// Returns 0, or -1 on a malformed argument.
+int dlion_oracle_worker_step(const dlion_oracle_segment* segs, uint32_t nseg,
+                             uint64_t d_pad, uint32_t n_workers, int gdtype,
+                             const void* g, float* m, uint32_t* packed,
+                             float beta1, float beta2, int nthreads) {
+    if (!segs || !g || !m || !packed || d_pad % 32 != 0 || n_workers == 0) return -1;
+    const uint64_t W = d_pad / 32;
+    const float om1 = 1.0f - beta1;   // R1: (1-beta) in binary32
+    const float om2 = 1.0f - beta2;
+    (void)nthreads;
+    for (uint32_t s = 0; s < nseg; ++s) {
+        const uint64_t lo = segs[s].elem_offset;
+        const uint64_t hi = lo + segs[s].numel;
+        if (hi > d_pad || lo % 32 != 0) return -1;      // no word is shared by two segments
+        if (hi == lo) continue;
+        const int64_t w_lo = static_cast<int64_t>(lo / 32);
+        const int64_t w_hi = static_cast<int64_t>((hi + 31) / 32);
+#pragma omp parallel for collapse(2) schedule(static) num_threads(nthreads > 0 ? nthreads : 1)
+        for (uint32_t i = 0; i < n_workers; ++i) {
+            for (int64_t w = w_lo; w < w_hi; ++w) {
+                uint32_t word = 0;
+                for (uint32_t b = 0; b < 32; ++b) {
+                    const uint64_t j = static_cast<uint64_t>(w) * 32 + b;
+                    if (j < lo || j >= hi) continue;            // padding bit stays 0
+                    const size_t idx = static_cast<size_t>(i) * d_pad + j;
+                    const float gf = load_grad(g, gdtype, idx);
+                    const float mo = m[idx];                    // R5: old momentum
+                    const float a1 = beta1 * mo;
+                    const float b1 = om1 * gf;
+                    const float c = a1 + b1;                    // Alg. 1, delta line
+                    word |= sign_bit(c) << b;
+                    const float a2 = beta2 * mo;
+                    const float b2 = om2 * gf;
+                    m[idx] = a2 + b2;                           // Alg. 1, momentum line
+                }
+                packed[static_cast<size_t>(i) * W + static_cast<size_t>(w)] = word;
+            }
+        }
+    }
+    return 0;
+}
+
+// Server side of Algorithm 1 followed by the parameter update of Section 3.2.
+//   packed     [N][d_pad/32]  the N binary vectors delta_{i,t}         (read)
+//   x          [d_pad]        parameters x_t -> x_{t+1}, f32           (in place)
+//   delta_bits [d_pad/32]     optional: Delta_t as bits (Majority Vote; for
+//                             Averaging it is sgn of the sum), padding bits 0
+//   count      [d_pad]        optional: P = number of +1 votes, u8 (N <= 255)
+// Returns 0, or -1 on a malformed argument.
+int dlion_oracle_aggregate_apply(const dlion_oracle_segment* segs, uint32_t nseg,
+                                 uint64_t d_pad, uint32_t n_workers, int mode,
+                                 const uint32_t* packed, float* x,
+                                 uint32_t* delta_bits, uint8_t* count,
+                                 float lr, float weight_decay, int nthreads) {
+    if (!segs || !packed || !x || d_pad % 32 != 0 || n_workers == 0) return -1;
+    if (count && n_workers > 255) return -1;
+    if (mode != DLION_ORACLE_MAJORITY && mode != DLION_ORACLE_AVERAGE) return -1;
+    const uint64_t W = d_pad / 32;
+    const int32_t N = static_cast<int32_t>(n_workers);
+    (void)nthreads;
+    for (uint32_t s = 0; s < nseg; ++s) {
+        const uint64_t lo = segs[s].elem_offset;
+        const uint64_t hi = lo + segs[s].numel;
+        if (hi > d_pad || lo % 32 != 0) return -1;
+        if (hi == lo) continue;
+        const int64_t w_lo = static_cast<int64_t>(lo / 32);
+        const int64_t w_hi = static_cast<int64_t>((hi + 31) / 32);
+#pragma omp parallel for schedule(static) num_threads(nthreads > 0 ? nthreads : 1)
+        for (int64_t w = w_lo; w < w_hi; ++w) {
+            uint32_t dword = 0;
+            for (uint32_t b = 0; b < 32; ++b) {
+                const uint64_t j = static_cast<uint64_t>(w) * 32 + b;
+                if (j < lo || j >= hi) continue;
+                int32_t P = 0;                                   // R4: +1 votes
+                for (int32_t i = 0; i < N; ++i) {
+                    P += static_cast<int32_t>((packed[static_cast<size_t>(i) * W + static_cast<size_t>(w)] >> b) & 1u);
+                }
+                const int32_t S = 2 * P - N;                     // S_t = sum_i delta_i
+                float Delta;
+                if (mode == DLION_ORACLE_AVERAGE) {
+                    Delta = static_cast<float>(S) / static_cast<float>(N);   // R6
+                } else {
+                    Delta = (S >= 0) ? 1.0f : -1.0f;             // R2, R3
+                }
+                if (S >= 0) dword |= 1u << b;
+                if (count) count[j] = static_cast<uint8_t>(P);
+                const float xo = x[j];
+                const float t1 = weight_decay * xo;
+                const float t2 = Delta + t1;
+                const float t3 = lr * t2;
+                x[j] = xo - t3;                                  // Section 3.2, last eq.
+            }
+            if (delta_bits) delta_bits[w] = dword;
+        }
+    }
+    return 0;
+}
+
+// Analytic communication volume per step in BITS (Table 1 and Section 3.2
+// "Communication Cost"), for d parameters and N workers.
+//   direction 0: all workers -> server, N * d (one bit per parameter per worker)
+//   direction 1: server -> one worker, d for Majority Vote; for Averaging an
+//                integer in {0..N} per parameter, which takes ceil(log2(N+1))
+//                bits (the paper rounds this to log N)
+uint64_t dlion_oracle_wire_bits(uint64_t d, uint32_t n_workers, int mode, int direction) {
+    if (direction == 0) return static_cast<uint64_t>(n_workers) * d;
+    if (mode == DLION_ORACLE_MAJORITY) return d;
+    uint32_t bits = 0;
+    while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;
+    return d * bits;
+}
+
+// 1 when this build honours the nthreads argument (OpenMP), else 0.
+int dlion_oracle_has_openmp(void) {
+#ifdef _OPENMP
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+}  // extern "C"

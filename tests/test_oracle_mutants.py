@@ -1,0 +1,54 @@
+"""Each plausible mistake, planted in a private copy of the oracle's source, must
+trip at least one pin.  The mistakes are planted on the CPU only."""
+import subprocess
+
+import pytest
+
+from oracle import dlion_oracle as orc
+from tests import oracle_pins
+
+MUTANTS = {
+    "delta_uses_beta2": ("const float a1 = beta1 * mo;", "const float a1 = beta2 * mo;"),
+    "delta_uses_om2": ("const float b1 = om1 * gf;", "const float b1 = om2 * gf;"),
+    "delta_uses_new_momentum": ("const float a1 = beta1 * mo;",
+                                "const float a1 = beta1 * (beta2 * mo + om2 * gf);"),
+    "delta_negated": ("word |= sign_bit(c) << b;", "word |= sign_bit(-c) << b;"),
+    "sign_of_zero_negative": ("return (v >= 0.0f) ? 1u : 0u;", "return (v > 0.0f) ? 1u : 0u;"),
+    "bit_order_reversed": ("word |= sign_bit(c) << b;", "word |= sign_bit(c) << (31 - b);"),
+    "momentum_uses_beta1": ("m[idx] = a2 + b2;", "m[idx] = a1 + b1;"),
+    "momentum_drops_gradient": ("m[idx] = a2 + b2;", "m[idx] = a2;"),
+    "one_minus_beta_dropped": ("const float om2 = 1.0f - beta2;", "const float om2 = 1.0f;"),
+    "tie_goes_negative": ("Delta = (S >= 0) ? 1.0f : -1.0f;", "Delta = (S > 0) ? 1.0f : -1.0f;"),
+    "sum_is_count": ("const int32_t S = 2 * P - N;", "const int32_t S = P;"),
+    "average_without_division": ("Delta = static_cast<float>(S) / static_cast<float>(N);",
+                                 "Delta = static_cast<float>(S);"),
+    "weight_decay_sign": ("const float t2 = Delta + t1;", "const float t2 = Delta - t1;"),
+    "weight_decay_dropped": ("const float t1 = weight_decay * xo;", "const float t1 = 0.0f * xo;"),
+    "update_sign": ("x[j] = xo - t3;", "x[j] = xo + t3;"),
+    "lr_outside_decay": ("const float t3 = lr * t2;", "const float t3 = lr * Delta + t1;"),
+    "only_first_worker_counted": ("P += static_cast<int32_t>((packed[static_cast<size_t>(i) * W",
+                                  "P += static_cast<int32_t>((packed[static_cast<size_t>(0) * W"),
+    "padding_written": ("if (j < lo || j >= hi) continue;            // padding bit stays 0",
+                        "if (j >= d_pad) continue;"),
+    "average_down_bits_floor_log": ("while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;",
+                                    "while ((2ull << bits) <= static_cast<uint64_t>(n_workers)) ++bits;"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_mutant_is_caught(name, tmp_path, oracle):
+    old, new = MUTANTS[name]
+    src = open(orc._SRC).read()
+    assert src.count(old) == 1, f"mutation site for {name} not found exactly once"
+    msrc = tmp_path / "mutant.cpp"
+    msrc.write_text(src.replace(old, new))
+    out = tmp_path / "libmutant.so"
+    subprocess.run(["g++", *orc.CXXFLAGS, "-o", str(out), str(msrc)], check=True)
+    lib = orc.load(str(out))
+    caught = []
+    for check in oracle_pins.ALL_CHECKS:
+        try:
+            check(lib)
+        except (AssertionError, ValueError):
+            caught.append(check.__name__)
+    assert caught, f"no pin notices the planted mistake '{name}'"
