@@ -1,0 +1,161 @@
+/*
+ * dlion.h -- C ABI of the Distributed-Lion optimizer step for NVIDIA B200 (sm_100a).
+ *
+ * One optimizer step of Distributed Lion (arXiv 2404.00438, Algorithm 1 and
+ * Section 3.2) over d parameters with N data-parallel workers, the N workers
+ * held as N state slices on one GPU:
+ *
+ *   worker i :  delta_i = sign(beta1 m_i + (1-beta1) g_i)      (old m_i)
+ *               m_i    <- beta2 m_i + (1-beta2) g_i
+ *               delta_i is packed 32 signs per uint32: the 1-bit wire buffer
+ *   server   :  S = sum_i delta_i ;  Delta = sign(S)  (Majority Vote)
+ *                                    Delta = S / N    (Averaging)
+ *   apply    :  x <- x - lr (Delta + lambda x)
+ *
+ * Conventions (the paper leaves them open; they are fixed here once):
+ *   - all arithmetic is IEEE binary32, one rounding per operation, no fused
+ *     multiply-add:  c = fl(fl(beta1*m) + fl((1-beta1)*g)), likewise m', and
+ *     x' = fl(x - fl(lr*fl(Delta + fl(lambda*x)))); (1-beta) is formed in binary32;
+ *     bf16 gradients are widened exactly;
+ *   - sign(v) = +1 when v >= 0 (either zero), -1 otherwise (NaN gives -1);
+ *   - an even-N tie (S = 0) gives Delta = +1 under Majority Vote;
+ *   - the server's integer is P = number of +1 votes in {0..N}; S = 2P - N;
+ *   - Averaging uses the correctly rounded quotient (float)(2P-N) / (float)N.
+ *
+ * Memory layout. Every buffer is DEVICE memory owned by the caller, unless a
+ * parameter says "host".  Arenas are flat and worker-major:
+ *     grads  [N][d_pad]     float or bf16 (dlion_gdtype)
+ *     m      [N][d_pad]     float
+ *     packed [N][d_pad/32]  uint32; bit b of word w is coordinate 32*w+b; 1 = "+1"
+ *     x      [d_pad]        float (all workers hold the same x, so one copy)
+ * A segment table names the coordinates that are parameters: segment k covers
+ * [elem_offset, elem_offset+numel).  elem_offset and d_pad are multiples of
+ * DLION_ALIGN (128) elements, segments are ascending and do not overlap.
+ * Coordinates outside every segment are padding: never read as parameters, never
+ * written; packed words that hold no parameter are never written, and padding
+ * bits inside a written word are 0.  Base pointers must be 16-byte aligned
+ * (count_out: 4-byte).
+ *
+ * Calls that launch work are asynchronous on the given CUDA stream (a
+ * cudaStream_t passed as void*; NULL = the default stream) and never
+ * synchronise.  The context's device must be current.  Nothing here throws,
+ * aborts or traps: every failure is a status code.  No CPU fallback exists.
+ */
+#ifndef DLION_H_
+#define DLION_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DLION_ALIGN 128u        /* elements: alignment of segment starts and of d_pad */
+#define DLION_MAX_WORKERS 255u  /* vote counts are kept in 8 bits */
+
+typedef struct dlion_ctx dlion_ctx; /* opaque; host-side object */
+
+typedef enum {
+    DLION_OK = 0,
+    DLION_EINVAL = 1, /* null pointer, value out of range, malformed segment table */
+    DLION_EALIGN = 2, /* a pointer or offset violates the alignment rules above */
+    DLION_ENOMEM = 3, /* host or device allocation failed */
+    DLION_ECUDA = 4,  /* a CUDA runtime call or a kernel launch reported an error */
+    DLION_ESTATE = 5  /* wrong device current, or context unusable */
+} dlion_status;
+
+typedef enum { DLION_MAJORITY = 0, DLION_AVERAGE = 1 } dlion_mode;
+typedef enum { DLION_GRAD_F32 = 0, DLION_GRAD_BF16 = 1 } dlion_gdtype;
+
+typedef struct {
+    uint64_t elem_offset; /* first coordinate, in elements, multiple of DLION_ALIGN */
+    uint64_t numel;       /* number of parameters (0 allowed) */
+} dlion_segment;
+
+/* Host-only check of a segment table against the layout rules above.
+ * Returns DLION_OK, DLION_EINVAL (null, nseg = 0, overlap, out of d_pad) or
+ * DLION_EALIGN (offset or d_pad not a multiple of DLION_ALIGN).  Touches no GPU. */
+dlion_status dlion_check_layout(const dlion_segment* segs, uint32_t nseg, uint64_t d_pad);
+
+/* Algorithm 1 "Inputs": N, beta1, beta2 in [0,1], learning rate eps >= 0, weight
+ * decay lambda >= 0, and the aggregation rule (Section 3.2).  Validates, then
+ * copies the segment table to the current device (a few bytes per segment; the
+ * only device memory the library owns).  *out is set only on DLION_OK.
+ * nseg = 1 with elem_offset = 0 describes a flat vector of d = numel. */
+dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nseg,
+                        uint64_t d_pad, uint32_t n_workers, float beta1, float beta2,
+                        float lr, float weight_decay, dlion_mode mode, dlion_gdtype gdtype);
+
+/* Learning-rate schedules (the paper's CIFAR runs use a cosine schedule,
+ * Section 5.1): sets eps for the following steps.  lr >= 0 and finite. */
+dlion_status dlion_set_lr(dlion_ctx* ctx, float lr);
+
+/* Worker side of Algorithm 1 (the two worker-side assignments; same equations
+ * in Section 3.2).  worker = -1: all N workers, pointers are the [N][...]
+ * arenas.  worker = i in [0,N): that worker only, pointers are ITS slices
+ * (grads[d_pad], m[d_pad], packed[d_pad/32]).
+ *   grads   in     gradients g_{i,t}
+ *   m       in/out momentum, updated in place
+ *   packed  out    delta_{i,t}, 1 bit per coordinate (Table 1: d bits per worker) */
+dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, float* m,
+                               uint32_t* packed, void* cuda_stream);
+
+/* Server side of Algorithm 1 (aggregate(S_t), Section 3.2) fused with the
+ * parameter update x <- x - eps (Delta + lambda x) (last equation of Section 3.2).
+ *   packed          in     [N][d_pad/32], the N binary vectors
+ *   x               in/out parameters, updated in place
+ *   delta_bits_out  out, nullable  [d_pad/32]: bit = (S >= 0), i.e. Delta of
+ *                   Majority Vote, the d-bit server->worker message of Table 1
+ *   count_out       out, nullable  [d_pad] bytes: P, the integer in {0..N} that
+ *                   Averaging sends back (Section 3.2 "Communication Cost") */
+dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float* x,
+                                   uint32_t* delta_bits_out, uint8_t* count_out,
+                                   void* cuda_stream);
+
+/* The whole of one Algorithm-1 iteration in ONE launch: a thread block holds a
+ * tile of coordinates for all N workers, votes in registers and applies x.
+ * Same results as dlion_worker_step(-1) followed by dlion_aggregate_apply.
+ *   packed_out  out, nullable: the wire buffer, if the caller still wants it. */
+dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, float* m, float* x,
+                              uint32_t* packed_out, void* cuda_stream);
+
+/* One whole step with the gradients in HOST memory (pinned memory makes the
+ * copies asynchronous).  Worker i's gradients are copied to the device while
+ * worker i-1's are being consumed by the worker-side kernel; after the last
+ * worker the server-side kernel runs and, if asked, Delta is copied back.
+ *   host_grads      in, host   [N][d_pad] gradients
+ *   m, x, packed    device     as above (packed is used as the wire buffer)
+ *   staging         device     2 * d_pad gradient elements (two slices)
+ *   delta_wire_dev  device, nullable  [d_pad/32] words (Majority Vote) or
+ *                   [d_pad] bytes (Averaging): Delta as the server sends it
+ *   host_delta_out  out, host, nullable: copy of delta_wire_dev; needs
+ *                   delta_wire_dev.  Complete when cuda_stream's work is.
+ * Uses one internal copy stream ordered against cuda_stream by events. */
+dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, float* m, float* x,
+                             uint32_t* packed, void* staging, void* delta_wire_dev,
+                             void* host_delta_out, void* cuda_stream);
+
+/* Analytic communication volume per step in bytes (Table 1; Section 3.2
+ * "Communication Cost"), d = number of parameters:
+ *   direction 0, all workers -> server:  N * d / 8
+ *   direction 1, server -> one worker:   d / 8 (Majority Vote), or
+ *                                        d * ceil(log2(N+1)) / 8 (Averaging)
+ *   direction 2: what one worker moves each way when fp32 gradients are
+ *                exchanged instead (Table 1, "Global Lion/AdamW": 32 d bits)
+ * Rounded up to whole bytes.  Returns 0 for a null context or bad direction. */
+uint64_t dlion_wire_bytes(const dlion_ctx* ctx, int direction);
+
+/* Number of kernels this context has launched so far. */
+uint64_t dlion_launch_count(const dlion_ctx* ctx);
+
+/* Static, human-readable name of a status code. */
+const char* dlion_status_str(dlion_status s);
+
+/* Frees the context and its device table.  Pending work must have completed. */
+void dlion_destroy(dlion_ctx* ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DLION_H_ */

@@ -1,0 +1,199 @@
+// C ABI of the library (include/dlion.h): argument checks, the context, and the
+// launches.  Everything that touches parameters runs in the kernels; this file
+// only validates, fills launch parameters and enqueues.
+#include <cmath>
+#include <cstdlib>
+#include <new>
+#include <vector>
+
+#include "dlion_ctx.cuh"
+
+namespace {
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bool unit_interval(float v) { return v >= 0.0f && v <= 1.0f; }           // false for NaN
+
+bool nonneg_finite(float v) { return v >= 0.0f && std::isfinite(v); }
+
+dlion::Betas betas_of(const dlion_ctx* c) {
+    dlion::Betas k;
+    k.b1 = c->beta1;
+    k.om1 = 1.0f - c->beta1;        // formed in binary32, as the contract says
+    k.b2 = c->beta2;
+    k.om2 = 1.0f - c->beta2;
+    return k;
+}
+
+dlion_status device_ok(const dlion_ctx* c) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
+    return dev == c->device ? DLION_OK : DLION_ESTATE;
+}
+
+}  // namespace
+
+extern "C" {
+
+dlion_status dlion_check_layout(const dlion_segment* segs, uint32_t nseg, uint64_t d_pad) {
+    if (segs == nullptr || nseg == 0 || d_pad == 0) return DLION_EINVAL;
+    if (d_pad % DLION_ALIGN != 0) return DLION_EALIGN;
+    uint64_t prev_end = 0;
+    for (uint32_t s = 0; s < nseg; ++s) {
+        if (segs[s].elem_offset % DLION_ALIGN != 0) return DLION_EALIGN;
+        if (segs[s].elem_offset < prev_end) return DLION_EINVAL;            // overlap or not ascending
+        if (segs[s].numel > d_pad || segs[s].elem_offset > d_pad - segs[s].numel) return DLION_EINVAL;
+        prev_end = segs[s].elem_offset + segs[s].numel;
+    }
+    return DLION_OK;
+}
+
+dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nseg, uint64_t d_pad,
+                        uint32_t n_workers, float beta1, float beta2, float lr, float weight_decay,
+                        dlion_mode mode, dlion_gdtype gdtype) {
+    if (out == nullptr) return DLION_EINVAL;
+    const dlion_status lay = dlion_check_layout(segs, nseg, d_pad);
+    if (lay != DLION_OK) return lay;
+    if (n_workers == 0 || n_workers > DLION_MAX_WORKERS) return DLION_EINVAL;
+    if (!unit_interval(beta1) || !unit_interval(beta2)) return DLION_EINVAL;
+    if (!nonneg_finite(lr) || !nonneg_finite(weight_decay)) return DLION_EINVAL;
+    if (mode != DLION_MAJORITY && mode != DLION_AVERAGE) return DLION_EINVAL;
+    if (gdtype != DLION_GRAD_F32 && gdtype != DLION_GRAD_BF16) return DLION_EINVAL;
+
+    dlion_ctx* c = new (std::nothrow) dlion_ctx;
+    if (c == nullptr) return DLION_ENOMEM;
+    std::vector<dlion::SegDev> rows;
+    try {
+        c->segs.assign(segs, segs + nseg);
+        rows.resize(nseg);
+    } catch (...) {
+        delete c;
+        return DLION_ENOMEM;
+    }
+    unsigned long long tiles = 0;
+    for (uint32_t s = 0; s < nseg; ++s) {
+        rows[s].elem_offset = segs[s].elem_offset;
+        rows[s].numel = segs[s].numel;
+        rows[s].first_tile = tiles;
+        tiles += (segs[s].numel + dlion::kTile - 1) / dlion::kTile;
+        c->d += segs[s].numel;
+    }
+    c->nseg = nseg;
+    c->ntiles = tiles;
+    c->d_pad = d_pad;
+    c->n_workers = n_workers;
+    c->beta1 = beta1;
+    c->beta2 = beta2;
+    c->lr = lr;
+    c->wd = weight_decay;
+    c->mode = mode;
+    c->gdtype = gdtype;
+
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    if (e != cudaSuccess) {
+        delete c;
+        return DLION_ECUDA;
+    }
+    e = cudaMalloc(reinterpret_cast<void**>(&c->segs_dev), sizeof(dlion::SegDev) * nseg);
+    if (e != cudaSuccess) {
+        delete c;
+        return e == cudaErrorMemoryAllocation ? DLION_ENOMEM : DLION_ECUDA;
+    }
+    e = cudaMemcpy(c->segs_dev, rows.data(), sizeof(dlion::SegDev) * nseg, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(c->segs_dev);
+        delete c;
+        return DLION_ECUDA;
+    }
+    *out = c;
+    return DLION_OK;
+}
+
+dlion_status dlion_set_lr(dlion_ctx* ctx, float lr) {
+    if (ctx == nullptr || !nonneg_finite(lr)) return DLION_EINVAL;
+    ctx->lr = lr;
+    return DLION_OK;
+}
+
+dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, float* m,
+                               uint32_t* packed, void* cuda_stream) {
+    if (ctx == nullptr || grads == nullptr || m == nullptr || packed == nullptr) return DLION_EINVAL;
+    if (worker < -1 || worker >= static_cast<int>(ctx->n_workers)) return DLION_EINVAL;
+    if (!aligned(grads, 16) || !aligned(m, 16) || !aligned(packed, 16)) return DLION_EALIGN;
+    const dlion_status ds = device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    dlion::WorkerParams p;
+    p.g = grads;
+    p.m = m;
+    p.packed = packed;
+    p.segs = ctx->segs_dev;
+    p.nseg = ctx->nseg;
+    p.n_workers = worker < 0 ? ctx->n_workers : 1u;
+    p.ntiles = ctx->ntiles;
+    p.d_pad = ctx->d_pad;
+    p.k = betas_of(ctx);
+    const cudaError_t e = dlion::launch_worker_step(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
+                                                    static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return DLION_ECUDA;
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float* x,
+                                   uint32_t* delta_bits_out, uint8_t* count_out, void* cuda_stream) {
+    if (ctx == nullptr || packed == nullptr || x == nullptr) return DLION_EINVAL;
+    if (!aligned(packed, 16) || !aligned(x, 16) || !aligned(delta_bits_out, 16) || !aligned(count_out, 4)) {
+        return DLION_EALIGN;
+    }
+    const dlion_status ds = device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    dlion::AggParams p;
+    p.packed = packed;
+    p.x = x;
+    p.delta_bits = delta_bits_out;
+    p.count = count_out;
+    p.segs = ctx->segs_dev;
+    p.nseg = ctx->nseg;
+    p.n_workers = ctx->n_workers;
+    p.ntiles = ctx->ntiles;
+    p.w_stride = ctx->d_pad / 32;
+    p.lr = ctx->lr;
+    p.wd = ctx->wd;
+    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    const cudaError_t e = dlion::launch_aggregate_apply(p, ctx->sm_count, static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return DLION_ECUDA;
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, float* m, float* x,
+                              uint32_t* packed_out, void* cuda_stream) {
+    if (ctx == nullptr || grads == nullptr || m == nullptr || x == nullptr) return DLION_EINVAL;
+    if (!aligned(grads, 16) || !aligned(m, 16) || !aligned(x, 16) || !aligned(packed_out, 16)) {
+        return DLION_EALIGN;
+    }
+    const dlion_status ds = device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    dlion::FusedParams p;
+    p.g = grads;
+    p.m = m;
+    p.x = x;
+    p.packed = packed_out;
+    p.segs = ctx->segs_dev;
+    p.nseg = ctx->nseg;
+    p.n_workers = ctx->n_workers;
+    p.ntiles = ctx->ntiles;
+    p.d_pad = ctx->d_pad;
+    p.k = betas_of(ctx);
+    p.lr = ctx->lr;
+    p.wd = ctx->wd;
+    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    const cudaError_t e = dlion::launch_step_fused(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
+                                                   static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return DLION_ECUDA;
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,151 @@
+// Shared declarations of the CUDA library: device-side segment table, the tile
+// lookup every kernel uses, and the pinned floating-point steps.
+//
+// Arithmetic contract (see include/dlion.h): binary32, one rounding per
+// operation, no fused multiply-add.  The _rn intrinsics below are never
+// contracted by the compiler, whatever -fmad says.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "dlion.h"
+
+namespace dlion {
+
+constexpr uint32_t kTile = 4096;        // coordinates per work item (all kernels)
+constexpr uint32_t kChunk = 128;        // coordinates one warp covers per vector access
+constexpr uint32_t kFull = 0xFFFFFFFFu;
+
+// One row per segment, in device memory.  first_tile is the running count of
+// tiles of the segments before it (a tile never spans two segments).
+struct SegDev {
+    unsigned long long elem_offset;
+    unsigned long long numel;
+    unsigned long long first_tile;
+};
+
+struct TileRef {
+    unsigned long long base;   // arena index of the tile's first coordinate
+    uint32_t valid;            // parameters in the tile, 1..kTile
+};
+
+// Largest s with segs[s].first_tile <= tile (segments with numel = 0 own no tile
+// and are never selected because the next row has the same first_tile).
+__device__ __forceinline__ TileRef find_tile(const SegDev* __restrict__ segs, uint32_t nseg,
+                                             unsigned long long tile) {
+    uint32_t lo = 0, hi = nseg;          // answer in [lo, hi)
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (__ldg(&segs[mid].first_tile) <= tile) lo = mid; else hi = mid;
+    }
+    const unsigned long long off = (tile - __ldg(&segs[lo].first_tile)) * kTile;
+    const unsigned long long left = __ldg(&segs[lo].numel) - off;
+    TileRef t;
+    t.base = __ldg(&segs[lo].elem_offset) + off;
+    t.valid = left < kTile ? static_cast<uint32_t>(left) : kTile;
+    return t;
+}
+
+// Algorithm 1, worker side, one coordinate: returns the sign bit of
+// beta1*m + (1-beta1)*g and replaces m by beta2*m + (1-beta2)*g (old m in both).
+struct Betas { float b1, om1, b2, om2; };
+
+__device__ __forceinline__ uint32_t lion_coord(float g, float& m, const Betas& k) {
+    const float c = __fadd_rn(__fmul_rn(k.b1, m), __fmul_rn(k.om1, g));
+    m = __fadd_rn(__fmul_rn(k.b2, m), __fmul_rn(k.om2, g));
+    return c >= 0.0f ? 1u : 0u;
+}
+
+// Section 3.2, last equation: x - lr*(Delta + lambda*x).
+__device__ __forceinline__ float apply_coord(float x, float delta, float lr, float wd) {
+    return __fsub_rn(x, __fmul_rn(lr, __fadd_rn(delta, __fmul_rn(wd, x))));
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t pair) { return __uint_as_float(pair & 0xFFFF0000u); }
+
+// Four consecutive gradients as floats, from fp32 or bf16 storage.
+template <bool BF16>
+__device__ __forceinline__ float4 load_grad4(const void* g, unsigned long long idx) {
+    if constexpr (BF16) {
+        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(g) + idx));
+        return make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+    } else {
+        return __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(g) + idx));
+    }
+}
+
+template <bool BF16>
+__device__ __forceinline__ float load_grad1(const void* g, unsigned long long idx) {
+    if constexpr (BF16) {
+        return __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(g)[idx]) << 16);
+    } else {
+        return static_cast<const float*>(g)[idx];
+    }
+}
+
+// Lane l of each group of 8 lanes holds a nibble (signs of coordinates 4l..4l+3
+// of a 32-coordinate word).  Returns the assembled word in all 8 lanes.
+__device__ __forceinline__ uint32_t gather_word(uint32_t nibble, uint32_t lane) {
+    uint32_t v = nibble << (4u * (lane & 7u));
+    v |= __shfl_xor_sync(kFull, v, 1);
+    v |= __shfl_xor_sync(kFull, v, 2);
+    v |= __shfl_xor_sync(kFull, v, 4);
+    return v;
+}
+
+// Bit k of a nibble -> byte k of a word (no carries: the four shifted copies do not overlap).
+__device__ __forceinline__ uint32_t spread_nibble(uint32_t nibble) {
+    return (nibble * 0x00204081u) & 0x01010101u;
+}
+
+// ---- launch parameters ----------------------------------------------------
+struct WorkerParams {
+    const void* g;
+    float* m;
+    uint32_t* packed;
+    const SegDev* segs;
+    uint32_t nseg;
+    uint32_t n_workers;              // workers this launch covers (1 for a single-worker call)
+    unsigned long long ntiles;       // tiles per worker
+    unsigned long long d_pad;        // elements between consecutive workers in g and m
+    Betas k;
+};
+
+struct AggParams {
+    const uint32_t* packed;
+    float* x;
+    uint32_t* delta_bits;            // nullable
+    uint8_t* count;                  // nullable
+    const SegDev* segs;
+    uint32_t nseg;
+    uint32_t n_workers;
+    unsigned long long ntiles;
+    unsigned long long w_stride;     // words between consecutive workers in packed
+    float lr, wd;
+    int average;                     // 0 = majority vote, 1 = averaging
+};
+
+struct FusedParams {
+    const void* g;
+    float* m;
+    float* x;
+    uint32_t* packed;                // nullable
+    const SegDev* segs;
+    uint32_t nseg;
+    uint32_t n_workers;
+    unsigned long long ntiles;
+    unsigned long long d_pad;
+    Betas k;
+    float lr, wd;
+    int average;
+};
+
+// Host-side launchers (one per .cu file).  grid = 0 asks the launcher to size a
+// persistent grid from the occupancy calculator and sm_count.
+cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s);
+cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s);
+cudaError_t launch_step_fused(const FusedParams& p, bool bf16, int sm_count, cudaStream_t s);
+
+}  // namespace dlion

@@ -1,0 +1,26 @@
+// The host-side context behind the opaque dlion_ctx of include/dlion.h.
+#pragma once
+
+#include <vector>
+
+#include "dlion_common.cuh"
+
+struct dlion_ctx {
+    std::vector<dlion_segment> segs;
+    dlion::SegDev* segs_dev = nullptr;
+    uint32_t nseg = 0;
+    unsigned long long ntiles = 0;
+    uint64_t d = 0;            // parameters
+    uint64_t d_pad = 0;
+    uint32_t n_workers = 0;
+    float beta1 = 0, beta2 = 0, lr = 0, wd = 0;
+    dlion_mode mode = DLION_MAJORITY;
+    dlion_gdtype gdtype = DLION_GRAD_F32;
+    int device = -1;
+    int sm_count = 0;
+    uint64_t launches = 0;
+    cudaStream_t copy_stream = nullptr;      // host-gradient pipeline (created on first use)
+    cudaEvent_t copied[2] = {nullptr, nullptr};
+    cudaEvent_t consumed[2] = {nullptr, nullptr};
+    cudaEvent_t entry = nullptr;
+};

@@ -1,0 +1,127 @@
+// Host-gradient step, analytic wire volume, and context teardown (include/dlion.h).
+#include "dlion_ctx.cuh"
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) % 16) == 0; }
+
+// Streams and events of the copy pipeline; created once, on first use.
+cudaError_t ensure_pipeline(dlion_ctx* c) {
+    if (c->copy_stream != nullptr) return cudaSuccess;
+    cudaError_t e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    for (int k = 0; k < 2 && e == cudaSuccess; ++k) {
+        e = cudaEventCreateWithFlags(&c->copied[k], cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->consumed[k], cudaEventDisableTiming);
+    }
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->entry, cudaEventDisableTiming);
+    return e;
+}
+
+}  // namespace
+
+extern "C" {
+
+dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, float* m, float* x,
+                             uint32_t* packed, void* staging, void* delta_wire_dev,
+                             void* host_delta_out, void* cuda_stream) {
+    if (ctx == nullptr || host_grads == nullptr || m == nullptr || x == nullptr || packed == nullptr ||
+        staging == nullptr) {
+        return DLION_EINVAL;
+    }
+    if (host_delta_out != nullptr && delta_wire_dev == nullptr) return DLION_EINVAL;
+    if (!aligned16(m) || !aligned16(x) || !aligned16(packed) || !aligned16(staging) ||
+        !aligned16(delta_wire_dev)) {
+        return DLION_EALIGN;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
+    if (dev != ctx->device) return DLION_ESTATE;
+    if (ensure_pipeline(ctx) != cudaSuccess) return DLION_ECUDA;
+
+    cudaStream_t main = static_cast<cudaStream_t>(cuda_stream);
+    const size_t gsz = ctx->gdtype == DLION_GRAD_BF16 ? 2 : 4;
+    const size_t slice = static_cast<size_t>(ctx->d_pad) * gsz;        // one worker's gradients
+    const size_t words = static_cast<size_t>(ctx->d_pad / 32);
+    const char* hsrc = static_cast<const char*>(host_grads);
+    char* stage = static_cast<char*>(staging);
+
+    // the copy stream may not start before the work already queued on main
+    // (a previous step may still be reading the staging slices)
+    if (cudaEventRecord(ctx->entry, main) != cudaSuccess) return DLION_ECUDA;
+    if (cudaStreamWaitEvent(ctx->copy_stream, ctx->entry, 0) != cudaSuccess) return DLION_ECUDA;
+
+    for (uint32_t i = 0; i < ctx->n_workers; ++i) {
+        const int b = static_cast<int>(i & 1u);
+        if (i >= 2 && cudaStreamWaitEvent(ctx->copy_stream, ctx->consumed[b], 0) != cudaSuccess) return DLION_ECUDA;
+        if (cudaMemcpyAsync(stage + b * slice, hsrc + i * slice, slice, cudaMemcpyHostToDevice,
+                            ctx->copy_stream) != cudaSuccess) return DLION_ECUDA;
+        if (cudaEventRecord(ctx->copied[b], ctx->copy_stream) != cudaSuccess) return DLION_ECUDA;
+        if (cudaStreamWaitEvent(main, ctx->copied[b], 0) != cudaSuccess) return DLION_ECUDA;
+        const dlion_status st = dlion_worker_step(ctx, static_cast<int>(i), stage + b * slice,
+                                                  m + static_cast<size_t>(i) * ctx->d_pad,
+                                                  packed + static_cast<size_t>(i) * words, main);
+        if (st != DLION_OK) return st;
+        if (cudaEventRecord(ctx->consumed[b], main) != cudaSuccess) return DLION_ECUDA;
+    }
+    const bool avg = ctx->mode == DLION_AVERAGE;
+    const dlion_status st = dlion_aggregate_apply(ctx, packed, x,
+                                                  avg ? nullptr : static_cast<uint32_t*>(delta_wire_dev),
+                                                  avg ? static_cast<uint8_t*>(delta_wire_dev) : nullptr, main);
+    if (st != DLION_OK) return st;
+    if (host_delta_out != nullptr) {
+        const size_t bytes = avg ? static_cast<size_t>(ctx->d_pad) : words * 4;
+        if (cudaMemcpyAsync(host_delta_out, delta_wire_dev, bytes, cudaMemcpyDeviceToHost, main) != cudaSuccess) {
+            return DLION_ECUDA;
+        }
+    }
+    return DLION_OK;
+}
+
+uint64_t dlion_wire_bytes(const dlion_ctx* ctx, int direction) {
+    if (ctx == nullptr) return 0;
+    const uint64_t d = ctx->d;
+    uint64_t bits;
+    if (direction == 0) {
+        bits = static_cast<uint64_t>(ctx->n_workers) * d;
+    } else if (direction == 1) {
+        uint32_t per = 1;
+        if (ctx->mode == DLION_AVERAGE) {
+            per = 0;
+            while ((1ull << per) < static_cast<uint64_t>(ctx->n_workers) + 1) ++per;   // N+1 values
+        }
+        bits = d * per;
+    } else if (direction == 2) {
+        bits = 32 * d;
+    } else {
+        return 0;
+    }
+    return (bits + 7) / 8;
+}
+
+uint64_t dlion_launch_count(const dlion_ctx* ctx) { return ctx == nullptr ? 0 : ctx->launches; }
+
+const char* dlion_status_str(dlion_status s) {
+    switch (s) {
+        case DLION_OK: return "ok";
+        case DLION_EINVAL: return "invalid argument";
+        case DLION_EALIGN: return "misaligned pointer or offset";
+        case DLION_ENOMEM: return "out of memory";
+        case DLION_ECUDA: return "CUDA error";
+        case DLION_ESTATE: return "wrong device or unusable context";
+    }
+    return "unknown status";
+}
+
+void dlion_destroy(dlion_ctx* ctx) {
+    if (ctx == nullptr) return;
+    if (ctx->segs_dev != nullptr) cudaFree(ctx->segs_dev);
+    for (int k = 0; k < 2; ++k) {
+        if (ctx->copied[k] != nullptr) cudaEventDestroy(ctx->copied[k]);
+        if (ctx->consumed[k] != nullptr) cudaEventDestroy(ctx->consumed[k]);
+    }
+    if (ctx->entry != nullptr) cudaEventDestroy(ctx->entry);
+    if (ctx->copy_stream != nullptr) cudaStreamDestroy(ctx->copy_stream);
+    delete ctx;
+}
+
+}  // extern "C"

@@ -1,0 +1,118 @@
+// Worker side of Algorithm 1 (arXiv 2404.00438): for every worker i and
+// coordinate j,
+//     delta_i[j] = sign(beta1 m_i[j] + (1-beta1) g_i[j])      (old m_i)
+//     m_i[j]    <- beta2 m_i[j] + (1-beta2) g_i[j]
+// with delta_i packed 32 signs per word into the 1-bit wire buffer
+// (Section 3.2, "Communication Cost": each worker sends d bits).
+//
+// A pure streaming kernel, bound by HBM: per coordinate and worker it reads the
+// gradient (2 or 4 B) and the momentum (4 B), writes the momentum (4 B) and 1/8 B
+// of signs.  Work item = (worker, tile of 4096 coordinates); a persistent grid
+// strides over the items.  Inside a tile each warp owns 512 consecutive
+// coordinates as four 128-coordinate chunks; lane l of a chunk holds coordinates
+// 4l..4l+3, so every load and store instruction of a warp is one contiguous run
+// (16 B per lane for fp32, 8 B per lane for bf16 gradients).  Eight lanes'
+// nibbles are merged into a word by three xor-shuffles, and the warp's 16 words
+// leave as one 64-byte run.
+#include "dlion_common.cuh"
+
+namespace dlion {
+namespace {
+
+constexpr int kThreads = 256;            // 8 warps x 512 coordinates = one tile
+constexpr int kChunksPerWarp = 4;
+
+template <bool BF16>
+__global__ void __launch_bounds__(kThreads)
+worker_step_kernel(const WorkerParams p) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp = threadIdx.x >> 5;
+    const unsigned long long n_items = p.ntiles * p.n_workers;
+    const unsigned long long w_stride = p.d_pad / 32;
+
+    for (unsigned long long item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const unsigned long long worker = item / p.ntiles;
+        const TileRef t = find_tile(p.segs, p.nseg, item - worker * p.ntiles);
+        const unsigned long long wbase = worker * p.d_pad;         // element offset of this worker
+        const uint32_t in_tile = warp * (kChunksPerWarp * kChunk); // first coordinate of this warp
+        uint32_t* words = p.packed + worker * w_stride + (t.base + in_tile) / 32;
+
+        if (t.valid == kTile) {
+            // ---- full tile: vector path, all loads issued before any use ----
+            const unsigned long long e0 = wbase + t.base + in_tile + lane * 4;
+            float4 g[kChunksPerWarp], m[kChunksPerWarp];
+#pragma unroll
+            for (int u = 0; u < kChunksPerWarp; ++u) {
+                g[u] = load_grad4<BF16>(p.g, e0 + u * kChunk);
+                m[u] = __ldcs(reinterpret_cast<const float4*>(p.m + e0 + u * kChunk));
+            }
+            uint32_t mine = 0;
+#pragma unroll
+            for (int u = 0; u < kChunksPerWarp; ++u) {
+                uint32_t nib = lion_coord(g[u].x, m[u].x, p.k);
+                nib |= lion_coord(g[u].y, m[u].y, p.k) << 1;
+                nib |= lion_coord(g[u].z, m[u].z, p.k) << 2;
+                nib |= lion_coord(g[u].w, m[u].w, p.k) << 3;
+                __stcs(reinterpret_cast<float4*>(p.m + e0 + u * kChunk), m[u]);
+                const uint32_t w = gather_word(nib, lane);
+                if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
+            }
+            // lane l (l%8 < 4) holds the word of chunk l%8, group l/8: word index 4*(l%8) + l/8
+            if ((lane & 7u) < kChunksPerWarp) words[4u * (lane & 7u) + (lane >> 3)] = mine;
+        } else {
+            // ---- last tile of a segment: per-coordinate guards -------------
+#pragma unroll 1
+            for (int u = 0; u < kChunksPerWarp; ++u) {
+                const uint32_t c0 = in_tile + u * kChunk;           // chunk start within the tile
+                if (c0 >= t.valid) break;                            // warp-uniform
+                const uint32_t j0 = c0 + lane * 4;
+                const unsigned long long e = wbase + t.base + j0;
+                uint32_t nib = 0;
+                if (j0 + 4 <= t.valid) {
+                    float4 g = load_grad4<BF16>(p.g, e);
+                    float4 m = __ldcs(reinterpret_cast<const float4*>(p.m + e));
+                    nib = lion_coord(g.x, m.x, p.k);
+                    nib |= lion_coord(g.y, m.y, p.k) << 1;
+                    nib |= lion_coord(g.z, m.z, p.k) << 2;
+                    nib |= lion_coord(g.w, m.w, p.k) << 3;
+                    __stcs(reinterpret_cast<float4*>(p.m + e), m);
+                } else {
+                    for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
+                        const float g = load_grad1<BF16>(p.g, e + q);
+                        float m = p.m[e + q];
+                        nib |= lion_coord(g, m, p.k) << q;
+                        p.m[e + q] = m;
+                    }
+                }
+                const uint32_t w = gather_word(nib, lane);
+                // only words that hold at least one parameter are written
+                if ((lane & 7u) == 0 && c0 + (lane >> 3) * 32 < t.valid) {
+                    words[4u * u + (lane >> 3)] = w;
+                }
+            }
+        }
+    }
+}
+
+template <bool BF16>
+cudaError_t launch(const WorkerParams& p, int sm_count, cudaStream_t s) {
+    int per_sm = 0;
+    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, worker_step_kernel<BF16>,
+                                                                  kThreads, 0);
+    if (e != cudaSuccess) return e;
+    if (per_sm < 1) per_sm = 1;
+    const unsigned long long n_items = p.ntiles * p.n_workers;
+    unsigned long long grid = static_cast<unsigned long long>(per_sm) * sm_count;
+    if (grid > n_items) grid = n_items;
+    if (grid == 0) return cudaSuccess;
+    worker_step_kernel<BF16><<<static_cast<unsigned>(grid), kThreads, 0, s>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s) {
+    return bf16 ? launch<true>(p, sm_count, s) : launch<false>(p, sm_count, s);
+}
+
+}  // namespace dlion

@@ -1,0 +1,166 @@
+"""Thin binding over the C ABI declared in ``include/dlion.h`` (same names).
+
+Argument marshalling only: tensors become device pointers, the current torch
+stream becomes the ``cudaStream_t``; every step of the optimizer runs in the CUDA
+library.  Importing this module loads ``libdlion.so`` and raises if it is
+missing: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+from . import build as _build
+
+MAJORITY, AVERAGE = 0, 1
+GRAD_F32, GRAD_BF16 = 0, 1
+ALIGN = 128
+MAX_WORKERS = 255
+OK, EINVAL, EALIGN, ENOMEM, ECUDA, ESTATE = range(6)
+
+EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_worker_step",
+           "dlion_aggregate_apply", "dlion_step_fused", "dlion_step_host", "dlion_wire_bytes",
+           "dlion_launch_count", "dlion_status_str", "dlion_destroy")
+
+
+class Segment(ctypes.Structure):
+    _fields_ = [("elem_offset", ctypes.c_uint64), ("numel", ctypes.c_uint64)]
+
+
+class DlionError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_str(status)} (status {status})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(_build.LIB):
+        raise ImportError(
+            f"{_build.LIB} is missing: build it with `python -m paper_2404_00438_b200.build` "
+            "(nvcc, sm_100a). This package has no CPU fallback.")
+    lib = ctypes.CDLL(_build.LIB)
+    vp, u32, u64, f32, i32 = (ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_float,
+                              ctypes.c_int)
+    seg_p = ctypes.POINTER(Segment)
+    lib.dlion_check_layout.argtypes = [seg_p, u32, u64]
+    lib.dlion_check_layout.restype = i32
+    lib.dlion_init.argtypes = [ctypes.POINTER(vp), seg_p, u32, u64, u32, f32, f32, f32, f32, i32, i32]
+    lib.dlion_init.restype = i32
+    lib.dlion_set_lr.argtypes = [vp, f32]
+    lib.dlion_set_lr.restype = i32
+    lib.dlion_worker_step.argtypes = [vp, i32, vp, vp, vp, vp]
+    lib.dlion_worker_step.restype = i32
+    lib.dlion_aggregate_apply.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.dlion_aggregate_apply.restype = i32
+    lib.dlion_step_fused.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.dlion_step_fused.restype = i32
+    lib.dlion_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.dlion_step_host.restype = i32
+    lib.dlion_wire_bytes.argtypes = [vp, i32]
+    lib.dlion_wire_bytes.restype = u64
+    lib.dlion_launch_count.argtypes = [vp]
+    lib.dlion_launch_count.restype = u64
+    lib.dlion_status_str.argtypes = [i32]
+    lib.dlion_status_str.restype = ctypes.c_char_p
+    lib.dlion_destroy.argtypes = [vp]
+    lib.dlion_destroy.restype = None
+    return lib
+
+
+_lib = _load()
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C library (for callers that want the raw ABI)."""
+    return _lib
+
+
+def status_str(status: int) -> str:
+    return _lib.dlion_status_str(int(status)).decode()
+
+
+def _seg_array(segments: Sequence[Tuple[int, int]]):
+    arr = (Segment * max(len(segments), 1))()
+    for k, (off, n) in enumerate(segments):
+        arr[k].elem_offset = int(off)
+        arr[k].numel = int(n)
+    return arr
+
+
+def check_layout(segments: Sequence[Tuple[int, int]], d_pad: int) -> int:
+    """``dlion_check_layout``: returns the status code (no exception)."""
+    return int(_lib.dlion_check_layout(_seg_array(segments), len(segments), int(d_pad)))
+
+
+def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Dlion:
+    """Owner of one ``dlion_ctx``.  Methods mirror the C calls one to one."""
+
+    def __init__(self, segments: Sequence[Tuple[int, int]], d_pad: int, n_workers: int,
+                 beta1: float = 0.9, beta2: float = 0.99, lr: float = 1e-4,
+                 weight_decay: float = 0.0, mode: int = MAJORITY, gdtype: int = GRAD_F32):
+        self._ctx = ctypes.c_void_p()
+        st = _lib.dlion_init(ctypes.byref(self._ctx), _seg_array(segments), len(segments), int(d_pad),
+                             int(n_workers), beta1, beta2, lr, weight_decay, int(mode), int(gdtype))
+        if st != OK:
+            self._ctx = ctypes.c_void_p()
+            raise DlionError(st, "dlion_init")
+        self.d_pad, self.n_workers, self.mode, self.gdtype = int(d_pad), int(n_workers), mode, gdtype
+
+    def _check(self, st: int, where: str) -> None:
+        if st != OK:
+            raise DlionError(st, where)
+
+    def set_lr(self, lr: float) -> None:
+        self._check(_lib.dlion_set_lr(self._ctx, lr), "dlion_set_lr")
+
+    def worker_step(self, worker: int, grads: torch.Tensor, m: torch.Tensor,
+                    packed: torch.Tensor) -> None:
+        self._check(_lib.dlion_worker_step(self._ctx, int(worker), _ptr(grads), _ptr(m), _ptr(packed),
+                                           _stream()), "dlion_worker_step")
+
+    def aggregate_apply(self, packed: torch.Tensor, x: torch.Tensor,
+                        delta_bits_out: Optional[torch.Tensor] = None,
+                        count_out: Optional[torch.Tensor] = None) -> None:
+        self._check(_lib.dlion_aggregate_apply(self._ctx, _ptr(packed), _ptr(x), _ptr(delta_bits_out),
+                                               _ptr(count_out), _stream()), "dlion_aggregate_apply")
+
+    def step_fused(self, grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor,
+                   packed_out: Optional[torch.Tensor] = None) -> None:
+        self._check(_lib.dlion_step_fused(self._ctx, _ptr(grads), _ptr(m), _ptr(x), _ptr(packed_out),
+                                          _stream()), "dlion_step_fused")
+
+    def step_host(self, host_grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor,
+                  packed: torch.Tensor, staging: torch.Tensor,
+                  delta_wire_dev: Optional[torch.Tensor] = None,
+                  host_delta_out: Optional[torch.Tensor] = None) -> None:
+        self._check(_lib.dlion_step_host(self._ctx, _ptr(host_grads), _ptr(m), _ptr(x), _ptr(packed),
+                                         _ptr(staging), _ptr(delta_wire_dev), _ptr(host_delta_out),
+                                         _stream()), "dlion_step_host")
+
+    def wire_bytes(self, direction: int) -> int:
+        return int(_lib.dlion_wire_bytes(self._ctx, int(direction)))
+
+    def launch_count(self) -> int:
+        return int(_lib.dlion_launch_count(self._ctx))
+
+    def destroy(self) -> None:
+        if self._ctx:
+            _lib.dlion_destroy(self._ctx)
+            self._ctx = ctypes.c_void_p()
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass

@@ -1,0 +1,174 @@
+"""CUDA library vs CPU oracle, element by element, through the C ABI (needs a B200)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2404_00438_b200 import inputs
+from tests import gpu_parity as gp
+
+pytestmark = pytest.mark.gpu
+
+MAJ, AVG = inputs.MAJORITY, inputs.AVERAGE
+RAGGED = [5, 200, 31, 32, 1, 4096, 4097, 8191, 12289, 0, 33, 128, 127]
+
+
+@pytest.fixture(scope="module")
+def dl():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    from paper_2404_00438_b200 import build
+    build.build()
+    from paper_2404_00438_b200 import dlion
+    return dlion
+
+
+# ---------------------------------------------------------------- config 1, ten steps
+@pytest.mark.parametrize("path", ["two_stage", "per_worker", "fused"])
+def test_c1_ten_steps(dl, path):
+    w = inputs.workload("c1")
+    worst = gp.run_small(dl, w, 10, path)
+    assert worst == 0, "pinned evaluation order should reproduce the oracle's fp32 state bit for bit"
+
+
+# ---------------------------------------------------------------- ragged tables, every N class
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 5, 7, 8, 15, 16, 33, 64, 127, 128, 255])
+@pytest.mark.parametrize("gd", ["f32", "bf16"])
+def test_ragged_segments(dl, n, gd):
+    scale = 1.0 if gd == "f32" else 1e-3
+    w = inputs.custom(RAGGED, n, MAJ, gd, scale=scale, lr=1e-3, weight_decay=0.5, zero_frac=0.02)
+    for path in ("two_stage", "fused"):
+        gp.run_small(dl, w, 3, path)
+    if n <= 8:
+        gp.run_small(dl, w, 2, "per_worker")
+
+
+def test_tiny_and_empty(dl):
+    for numels in ([1], [31], [32], [33], [1000], [0, 0, 7], [0]):
+        for n in (1, 2, 5):
+            w = inputs.custom(numels, n, MAJ, "f32")
+            for path in ("two_stage", "fused", "per_worker"):
+                gp.run_small(dl, w, 2, path)
+
+
+def test_multi_tile_with_ragged_tail(dl):
+    w = inputs.custom([3 * 4096 * 160 + 1234, 777], 4, AVG, "bf16", scale=1e-3, lr=1e-3, weight_decay=1.0)
+    for path in ("two_stage", "fused"):
+        assert gp.run_small(dl, w, 3, path) == 0
+
+
+# ---------------------------------------------------------------- degenerate values
+def test_special_values(dl):
+    """+-0, exact cancellation beta1*m = -(1-beta1)*g, NaN, +-Inf, denormals, |x| > 1/lambda."""
+    n, d = 4, 4096 + 640
+    w = inputs.custom([d], n, MAJ, "f32", beta1=0.5, beta2=0.75, lr=0.25, weight_decay=0.5)
+    rng = np.random.default_rng(11)
+    specials = np.array([0.0, -0.0, 1.0, -1.0, np.nan, np.inf, -np.inf, 1e-42, -1e-42, 3e38, -3e38,
+                         1.1754944e-38], np.float32)
+    m0 = rng.choice(specials, size=(n, w.d_pad)).astype(np.float32)
+    g0 = rng.choice(specials, size=(n, w.d_pad)).astype(np.float32)
+    g0[:, :512] = -m0[:, :512]                       # beta1 = 1/2: c = 0.5 m - 0.5 m = +-0 -> +1
+    x0 = (rng.standard_normal(w.d_pad) * 5).astype(np.float32)
+    g1 = rng.standard_normal((n, w.d_pad)).astype(np.float32)
+    for a in (m0, g0, g1):
+        a[:, d:] = 0
+    x0[d:] = 0
+    grads = [torch.from_numpy(g0), torch.from_numpy(g1)]
+    for path in ("two_stage", "fused"):
+        gp.run_small(dl, w, 2, path, m0=torch.from_numpy(m0), x0=torch.from_numpy(x0), grads=grads)
+
+
+def test_even_n_ties_are_positive(dl):
+    n, d = 6, 4096
+    w = inputs.custom([d], n, MAJ, "f32", beta1=0.0, beta2=0.0, lr=1.0, weight_decay=0.0)
+    g = torch.ones(n, w.d_pad)
+    g[: n // 2] = -1.0                               # exact tie on every coordinate
+    dev = torch.device("cuda:0")
+    ctx = gp.make_ctx(dl, w)
+    m = torch.zeros(n, w.d_pad, device=dev)
+    x = torch.zeros(w.d_pad, device=dev)
+    packed = torch.zeros(n, w.d_pad // 32, dtype=torch.int32, device=dev)
+    dbits = torch.zeros(w.d_pad // 32, dtype=torch.int32, device=dev)
+    ctx.worker_step(-1, g.to(dev), m, packed)
+    ctx.aggregate_apply(packed, x, dbits)
+    torch.cuda.synchronize()
+    assert bool((x == -1.0).all()) and bool((dbits == -1).all())
+    gp.run_small(dl, w, 1, "two_stage", grads=[g])
+    ctx.destroy()
+
+
+def test_set_lr_and_launch_count(dl):
+    w = inputs.custom([5000], 3, AVG, "f32", lr=0.5, weight_decay=0.0)
+    dev = torch.device("cuda:0")
+    ctx = gp.make_ctx(dl, w)
+    g = inputs.fill_grads(w, 0, torch.empty(3, w.d_pad)).to(dev)
+    m = torch.zeros(3, w.d_pad, device=dev)
+    packed = torch.zeros(3, w.d_pad // 32, dtype=torch.int32, device=dev)
+    x1 = torch.zeros(w.d_pad, device=dev)
+    x2 = torch.zeros(w.d_pad, device=dev)
+    assert ctx.launch_count() == 0
+    ctx.worker_step(-1, g, m, packed)
+    ctx.aggregate_apply(packed, x1)
+    ctx.set_lr(0.25)
+    ctx.aggregate_apply(packed, x2)
+    torch.cuda.synchronize()
+    assert ctx.launch_count() == 3
+    assert torch.equal(x1, 2 * x2)                   # lambda = 0: x' = -lr * Delta
+    d = w.d
+    assert ctx.wire_bytes(0) == (3 * d + 7) // 8 and ctx.wire_bytes(1) == (2 * d + 7) // 8
+    assert ctx.wire_bytes(2) == 4 * d and ctx.wire_bytes(3) == 0
+    ctx.destroy()
+
+
+def test_argument_errors_with_a_context(dl):
+    w = inputs.custom([5000], 2, MAJ, "f32")
+    dev = torch.device("cuda:0")
+    ctx = gp.make_ctx(dl, w)
+    g = torch.zeros(2, w.d_pad, device=dev)
+    m = torch.zeros(2, w.d_pad, device=dev)
+    x = torch.zeros(w.d_pad + 4, device=dev)
+    packed = torch.zeros(2, w.d_pad // 32, dtype=torch.int32, device=dev)
+    for bad_worker in (-2, 2):
+        with pytest.raises(dl.DlionError) as e:
+            ctx.worker_step(bad_worker, g, m, packed)
+        assert e.value.status == dl.EINVAL
+    with pytest.raises(dl.DlionError) as e:
+        ctx.aggregate_apply(packed, x[1:])           # 4-byte aligned only
+    assert e.value.status == dl.EALIGN
+    with pytest.raises(dl.DlionError) as e:
+        ctx.worker_step(-1, g.view(-1)[1:], m, packed)
+    assert e.value.status == dl.EALIGN
+    raw = dl.lib()
+    assert raw.dlion_worker_step(ctx._ctx, -1, None, m.data_ptr(), packed.data_ptr(), None) == dl.EINVAL
+    assert raw.dlion_step_host(ctx._ctx, g.data_ptr(), m.data_ptr(), x.data_ptr(), packed.data_ptr(),
+                               g.data_ptr(), None, g.data_ptr(), None) == dl.EINVAL
+    ctx.worker_step(-1, g, m, packed)                # the context is still usable
+    torch.cuda.synchronize()
+    ctx.destroy()
+
+
+# ---------------------------------------------------------------- host-gradient step
+@pytest.mark.parametrize("mode", [MAJ, AVG])
+def test_step_host_matches_oracle(dl, mode):
+    w = inputs.custom([70000, 333], 5, mode, "bf16", scale=1e-3, lr=1e-3, weight_decay=1.0)
+    dev = torch.device("cuda:0")
+    N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
+    ctx = gp.make_ctx(dl, w)
+    x0 = inputs.fill_x0(w, torch.empty(D))
+    ora = gp.OracleState(w, 0, D, np.zeros((N, D), np.float32), x0.numpy(), [mode])
+    m = torch.zeros(N, D, device=dev)
+    x = x0.to(dev)
+    packed = torch.zeros(N, W, dtype=torch.int32, device=dev)
+    staging = torch.empty(2, D, dtype=torch.bfloat16, device=dev)
+    wire = torch.zeros(D if mode == AVG else W * 4, dtype=torch.uint8, device=dev)
+    host_wire = torch.zeros(wire.shape, dtype=torch.uint8).pin_memory()
+    host_g = torch.empty(N, D, dtype=torch.bfloat16).pin_memory()
+    for t in range(4):
+        inputs.fill_grads(w, t, host_g)
+        ora.step(inputs.as_numpy_grads(host_g))
+        ctx.step_host(host_g, m, x, packed, staging, wire, host_wire)
+        torch.cuda.synchronize()
+        gp.compare("packed", packed.cpu().numpy().view(np.uint32), ora.packed, True)
+        gp.compare("m", m.cpu().numpy(), ora.m, False)
+        gp.compare("x", x.cpu().numpy(), ora.x[mode], False)
+        want = ora.count[mode] if mode == AVG else ora.dbits[mode].view(np.uint8)
+        gp.compare("wire", host_wire.numpy(), want, True)
+    ctx.destroy()
