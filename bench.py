@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the Distributed-Lion optimizer step (arXiv 2404.00438) on B200.
+
+One "step" is one pass of the whole hot path over one batch of synthetic
+gradients: the worker-side kernel for all N workers (sign + pack + momentum),
+then the server-side kernel (vote / average + parameter update).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c5] [--mode majority]
+    python bench.py --impl reference ...      # the CPU oracle on a bounded sample
+
+Prints ONE JSON line on rank 0.  Timing is by CUDA events on the launching
+stream; every input is seeded and synthetic.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2404_00438_b200 import inputs  # noqa: E402
+
+METRIC = "dlion_step_param_worker_updates_per_s"
+UNIT = "G param*worker updates/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch of the worker-side kernel from an ncu capture
+# (dram__bytes_read.sum + dram__bytes_write.sum), as bytes per param*worker, keyed
+# by the SHA-256 of the kernel's source at capture time: reported only while the
+# source is unchanged.  See profiles/.
+NCU_TRAFFIC = {}
+
+
+def kernel_hash() -> str:
+    h = hashlib.sha256()
+    for name in ("worker_step.cu", "dlion_common.cuh"):
+        h.update(open(os.path.join(ROOT, "paper_2404_00438_b200", "csrc", name), "rb").read())
+    return h.hexdigest()[:16]
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi polled every 200 ms while the timed region runs (read-only)."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, reasons, smax, power = [], set(), None, []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            f = [v.strip() for v in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax = float(f[2])
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=smax, reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return out
+
+
+def bytes_per_param_worker_k1(w) -> float:
+    """Worker-side kernel: gradient + momentum read + momentum write + 1/8 B of signs."""
+    return w.grad_bytes + 4 + 4 + 1 / 8
+
+
+def bytes_per_param_k2(w) -> float:
+    """Server-side kernel: N/8 B of votes + parameter read + write."""
+    return w.n_workers / 8 + 4 + 4
+
+
+def mode_of(name: str) -> int:
+    return {"majority": inputs.MAJORITY, "average": inputs.AVERAGE}[name]
+
+
+def oracle_sample_rate(w, mode: int, seconds: float, nthreads: int):
+    """Times the CPU oracle (as it stands) on a bounded sample: the first 2^20
+    arena coordinates of the workload, all N workers, repeated steps."""
+    from oracle import dlion_oracle as orc
+    orc.build()
+    n = min(w.d_pad, 1 << 20)
+    segs = []
+    for off, cnt in w.segments:
+        a, b = off, min(off + cnt, n)
+        if a < b:
+            segs.append((a, b - a))
+    params = sum(c for _, c in segs)
+    g = inputs.as_numpy_grads(inputs.fill_grads(w, 0, torch.empty(w.n_workers, n, dtype=inputs.grad_torch_dtype(w)),
+                                               0, n))
+    m = np.zeros((w.n_workers, n), np.float32)
+    x = inputs.fill_x0(w, torch.empty(n), 0, n).numpy()
+    packed = np.zeros((w.n_workers, n // 32), np.uint32)
+
+    def one():
+        orc.worker_step(segs, n, w.n_workers, g, m, packed, w.beta1, w.beta2, nthreads=nthreads)
+        orc.aggregate_apply(segs, n, w.n_workers, mode, packed, x, w.lr, w.weight_decay, nthreads=nthreads)
+
+    one()                                   # warm-up, page faults
+    t0 = time.perf_counter()
+    one()
+    dt = time.perf_counter() - t0
+    steps = max(1, min(200, int(seconds / max(dt, 1e-6))))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    dt = time.perf_counter() - t0
+    rate = params * w.n_workers * steps / dt / 1e9
+    sample = (f"first {n} arena coordinates ({params} parameters) of {w.name}, all {w.n_workers} workers, "
+              f"{steps} steps, {dt:.1f} s")
+    return rate, sample, steps, dt
+
+
+def run_reference(args):
+    """The oracle, as it stands, on the host cores: bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    w = inputs.workload(args.workload)
+    mode = mode_of(args.mode) if args.mode else w.mode
+    cores = os.cpu_count() or 1
+    for _ in range(max(args.warmup, 0)):
+        oracle_sample_rate(w, mode, 0.0, cores)
+    rates, secs, sample = [], 0.0, ""
+    for _ in range(args.steps):
+        r, sample, _, dt = oracle_sample_rate(w, mode, 2.0, cores)
+        rates.append(r)
+        secs += dt
+    value = statistics.mean(rates)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / max(args.steps, 1),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "n_workers": w.n_workers, "d": w.d,
+                   "mode": "average" if mode else "majority", "grads": w.grad_dtype},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": "each step: " + sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import torch.distributed as dist
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2404_00438_b200 import build, dlion
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+
+    w = inputs.workload(args.workload)
+    if args.n_workers:
+        w.n_workers = args.n_workers
+    w.seed += rank                                    # each rank owns a different slab of a larger model
+    mode = mode_of(args.mode) if args.mode else w.mode
+    N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
+    gdt = inputs.grad_torch_dtype(w)
+    ctx = dlion.Dlion(w.segments, D, N, w.beta1, w.beta2, w.lr, w.weight_decay, mode,
+                      dlion.GRAD_F32 if w.grad_dtype == "f32" else dlion.GRAD_BF16)
+    g = torch.empty(N, D, dtype=gdt, device=dev)
+    m = torch.zeros(N, D, device=dev)
+    x = inputs.fill_x0(w, torch.empty(D, device=dev))
+    packed = torch.zeros(N, W, dtype=torch.int32, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step():
+        if args.path == "fused":
+            ctx.step_fused(g, m, x, None)
+        else:
+            ctx.worker_step(-1, g, m, packed)
+            ctx.aggregate_apply(packed, x)
+
+    for t in range(args.warmup):
+        inputs.fill_grads(w, t, g)
+        step()
+    barrier()
+
+    # ---- timed region: K steps, fresh gradients generated between steps (untimed)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.launch_count()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for t in range(args.steps):
+        inputs.fill_grads(w, args.warmup + t, g)
+        barrier()
+        ev[t][0].record(stream)
+        if args.path == "fused":
+            ctx.step_fused(g, m, x, None)
+            ev[t][1].record(stream)
+        else:
+            ctx.worker_step(-1, g, m, packed)
+            ev[t][1].record(stream)
+            ctx.aggregate_apply(packed, x)
+        ev[t][2].record(stream)
+    barrier()
+    launches = ctx.launch_count() - launches0
+    k1_ms = [e[0].elapsed_time(e[1]) for e in ev]
+    k2_ms = [e[1].elapsed_time(e[2]) for e in ev]
+    total_ms = sum(e[0].elapsed_time(e[2]) for e in ev)
+
+    # ---- the same K steps back to back on the last gradients (sustained clocks)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    b2b_ms = e0.elapsed_time(e1) / args.steps
+    clocks = sampler.stop() if rank == 0 else None
+
+    t_all = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t_all, op=dist.ReduceOp.MAX)
+    total_ms_max = float(t_all.item())
+    units = w.d * N * args.steps * world               # param*worker updates, all ranks
+    value = units / (total_ms_max * 1e-3) / 1e9
+
+    # ---- end to end: gradients in pinned host memory, Delta read back
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, ctx, w, mode, g, m, x, packed, dev, world, barrier)
+
+    if rank == 0:
+        peak, peak_src = measured_peak()
+        k1 = statistics.mean(k1_ms)
+        k2 = statistics.mean(k2_ms)
+        if args.path == "fused":
+            alg_bytes = w.d * (N * (w.grad_bytes + 8) + 8)
+            name = "step_fused_kernel"
+        else:
+            alg_bytes = w.d * N * bytes_per_param_worker_k1(w)
+            name = "worker_step_kernel"
+        achieved = alg_bytes / (k1 * 1e-3) / 1e9
+        traffic = NCU_TRAFFIC.get((name, kernel_hash()))
+        roofline = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_source": peak_src, "frac_of_8tbs_nominal": achieved / 8000.0,
+                    "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": k1,
+                    "traffic": None if traffic is None else traffic * w.d * N}
+        stages = None
+        if args.path != "fused":
+            b2 = w.d * bytes_per_param_k2(w)
+            stages = {"aggregate_apply_kernel": {"achieved": b2 / (k2 * 1e-3) / 1e9, "unit": "GB/s",
+                                                 "frac": b2 / (k2 * 1e-3) / 1e9 / peak, "ms_per_launch": k2,
+                                                 "algorithmic_bytes_per_launch": b2}}
+        cpu = None
+        if not args.no_cpu_baseline and world == 1:
+            cores = os.cpu_count() or 1
+            rate, sample, _, _ = oracle_sample_rate(w, mode, args.cpu_seconds, cores)
+            cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+        up, down = ctx.wire_bytes(0), ctx.wire_bytes(1)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": args.workload, "n_workers": N, "d": w.d, "grads": w.grad_dtype,
+                       "mode": "average" if mode else "majority", "path": args.path,
+                       "l2": "inputs larger than L2 (no flush needed)" if N * D * (w.grad_bytes + 4) > 4 * 126e6
+                             else "working set comparable to L2: latency-bound case",
+                       "grads_per_step": "fresh seeded gradients generated between timed steps, untimed",
+                       "per_rank": "each rank steps its own full-size coordinate slab; no collective"},
+            "ms_per_step_back_to_back": b2b_ms,
+            "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": launches, "clocks": clocks,
+            "wire_bytes_per_step": {"up_all_workers": up, "down_per_worker": down,
+                                    "fp32_gradients_each_way_per_worker": ctx.wire_bytes(2),
+                                    "fp32_ring_allreduce_per_gpu": int(2 * (N - 1) / N * 4 * w.d)},
+        }
+        print(json.dumps(line), flush=True)
+    ctx.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, ctx, w, mode, g, m, x, packed, dev, world, barrier):
+    """dlion_step_host: per step, N*D gradient elements host->device, Delta device->host."""
+    import torch.distributed as dist
+    N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
+    host_g = torch.empty(N, D, dtype=g.dtype).pin_memory()
+    host_g.copy_(g)
+    staging = torch.empty(2, D, dtype=g.dtype, device=dev)
+    wire_bytes = D if mode == inputs.AVERAGE else W * 4
+    wire = torch.zeros(wire_bytes, dtype=torch.uint8, device=dev)
+    host_wire = torch.zeros(wire_bytes, dtype=torch.uint8).pin_memory()
+    stream = torch.cuda.current_stream()
+    for _ in range(args.e2e_warmup):
+        ctx.step_host(host_g, m, x, packed, staging, wire, host_wire)
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.e2e_steps):
+        ctx.step_host(host_g, m, x, packed, staging, wire, host_wire)
+    e1.record(stream)
+    barrier()
+    t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item()) / args.e2e_steps
+    del host_g, staging
+    return {"value": w.d * N * world / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+            "steps": args.e2e_steps, "h2d_bytes_per_step": N * D * w.grad_bytes,
+            "d2h_bytes_per_step": wire_bytes, "call": "dlion_step_host (pinned host gradients in, Delta out)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--n-workers", type=int, default=0, help="override N (the c4 sweep)")
+    ap.add_argument("--mode", default=None, choices=["majority", "average"])
+    ap.add_argument("--path", default="two_stage", choices=["two_stage", "fused"])
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-warmup", type=int, default=1)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3                               # timing hygiene: at least three warm-up steps
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
