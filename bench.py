@@ -125,11 +125,11 @@ def mode_of(name: str) -> int:
 
 
 def oracle_sample_rate(w, mode: int, seconds: float, nthreads: int):
-    """Times the CPU oracle (as it stands) on a bounded sample: the first 2^20
+    """Times the CPU oracle (as it stands) on a bounded sample: the first 2^22
     arena coordinates of the workload, all N workers, repeated steps."""
     from oracle import dlion_oracle as orc
     orc.build()
-    n = min(w.d_pad, 1 << 20)
+    n = min(w.d_pad, 1 << 22)
     segs = []
     for off, cnt in w.segments:
         a, b = off, min(off + cnt, n)
@@ -150,7 +150,7 @@ def oracle_sample_rate(w, mode: int, seconds: float, nthreads: int):
     t0 = time.perf_counter()
     one()
     dt = time.perf_counter() - t0
-    steps = max(1, min(200, int(seconds / max(dt, 1e-6))))
+    steps = max(1, min(5000, int(seconds / max(dt, 1e-6))))
     t0 = time.perf_counter()
     for _ in range(steps):
         one()
