@@ -53,6 +53,7 @@ extern "C" {
 
 #define DLION_ALIGN 128u        /* elements: alignment of segment starts and of d_pad */
 #define DLION_MAX_WORKERS 255u  /* vote counts are kept in 8 bits */
+#define DLION_STATIC_MAX_COORD_WORKERS 134217728ull /* dlion_step_static: limit on N * d_pad */
 
 typedef struct dlion_ctx dlion_ctx; /* opaque; host-side object */
 
@@ -135,6 +136,33 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, float* m, float
 dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, float* m, float* x,
                              uint32_t* packed, void* staging, void* delta_wire_dev,
                              void* host_delta_out, void* cuda_stream);
+
+/* (No counterpart in the paper: an entry point for callers that cannot allocate.)
+ * One two-stage step -- the worker-side kernel for all N workers, then the
+ * server-side kernel -- on a flat vector of d parameters, without dlion_init and
+ * without a caller-supplied wire buffer.  It is meant for callers that must not
+ * call cudaMalloc where they step the optimizer: a host whose allocator already
+ * owns all device memory, a latency-critical loop that cannot take cudaMalloc's
+ * device-wide synchronisation, or a plug-in restricted to the buffers it is
+ * handed.  The segment table and the 1-bit wire buffer live in a fixed array
+ * inside the library image (16 MiB + 256 B per GPU that loads the library, held
+ * until the process exits).  The call allocates nothing, on host or device.
+ *   d, n_workers   the problem; d_pad = d rounded up to DLION_ALIGN, and
+ *                  n_workers * d_pad <= DLION_STATIC_MAX_COORD_WORKERS, else
+ *                  DLION_EINVAL ("does not fit the fixed scratch")
+ *   grads [N][d_pad], m [N][d_pad] (in/out), x [d_pad] (in/out): device, 16-byte
+ *                  aligned, as for dlion_worker_step(-1) / dlion_aggregate_apply
+ * Results are those of dlion_worker_step(-1) + dlion_aggregate_apply with the
+ * same hyper-parameters.  The first call on each device looks up the array's
+ * device address (that device must be current); make that first call before
+ * any stream capture begins.  All calls on a device share the array and it keeps
+ * the last call's bits: every word the step reads is rewritten first, so nothing
+ * needs clearing, but two calls that overlap on the GPU (different streams, no
+ * ordering) race on it and give undefined results. */
+dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float beta1, float beta2,
+                               float lr, float weight_decay, dlion_mode mode,
+                               dlion_gdtype gdtype, const void* grads, float* m, float* x,
+                               void* cuda_stream);
 
 /* Analytic communication volume per step in bytes (Table 1; Section 3.2
  * "Communication Cost"), d = number of parameters:

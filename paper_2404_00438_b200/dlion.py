@@ -22,7 +22,8 @@ MAX_WORKERS = 255
 OK, EINVAL, EALIGN, ENOMEM, ECUDA, ESTATE = range(6)
 
 EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_worker_step",
-           "dlion_aggregate_apply", "dlion_step_fused", "dlion_step_host", "dlion_wire_bytes",
+           "dlion_aggregate_apply", "dlion_step_fused", "dlion_step_host", "dlion_step_static",
+           "dlion_wire_bytes",
            "dlion_launch_count", "dlion_status_str", "dlion_destroy")
 
 
@@ -59,6 +60,8 @@ def _load() -> ctypes.CDLL:
     lib.dlion_step_fused.restype = i32
     lib.dlion_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.dlion_step_host.restype = i32
+    lib.dlion_step_static.argtypes = [u64, u32, f32, f32, f32, f32, i32, i32, vp, vp, vp, vp]
+    lib.dlion_step_static.restype = i32
     lib.dlion_wire_bytes.argtypes = [vp, i32]
     lib.dlion_wire_bytes.restype = u64
     lib.dlion_launch_count.argtypes = [vp]
@@ -93,6 +96,21 @@ def _seg_array(segments: Sequence[Tuple[int, int]]):
 def check_layout(segments: Sequence[Tuple[int, int]], d_pad: int) -> int:
     """``dlion_check_layout``: returns the status code (no exception)."""
     return int(_lib.dlion_check_layout(_seg_array(segments), len(segments), int(d_pad)))
+
+
+STATIC_MAX_COORD_WORKERS = 134217728
+
+
+def step_static(d: int, n_workers: int, beta1: float, beta2: float, lr: float, weight_decay: float,
+                mode: int, gdtype: int, grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor) -> None:
+    """``dlion_step_static``: one two-stage step on a flat vector for callers that cannot
+    allocate device memory (no context, no wire buffer: both live in a fixed array inside the
+    library, shared by all calls on the device).  Raises DlionError when N * d_pad exceeds
+    STATIC_MAX_COORD_WORKERS."""
+    st = _lib.dlion_step_static(int(d), int(n_workers), beta1, beta2, lr, weight_decay, int(mode),
+                                int(gdtype), _ptr(grads), _ptr(m), _ptr(x), _stream())
+    if st != OK:
+        raise DlionError(st, "dlion_step_static")
 
 
 def _ptr(t: Optional[torch.Tensor]) -> Optional[int]:
