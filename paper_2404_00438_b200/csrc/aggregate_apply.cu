@@ -169,31 +169,25 @@ aggregate_apply_kernel(const AggParams p) {
 }
 
 template <int PLANES>
-cudaError_t launch(const AggParams& p, int sm_count, cudaStream_t s) {
-    int per_sm = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, aggregate_apply_kernel<PLANES>,
-                                                                  kThreads, 0);
-    if (e != cudaSuccess) return e;
-    if (per_sm < 1) per_sm = 1;
-    unsigned long long grid = static_cast<unsigned long long>(per_sm) * sm_count;
-    if (grid > p.ntiles) grid = p.ntiles;
-    if (grid == 0) return cudaSuccess;
-    aggregate_apply_kernel<PLANES><<<static_cast<unsigned>(grid), kThreads, 0, s>>>(p);
+cudaError_t launch(const AggParams& p, cudaStream_t s) {
+    if (p.ntiles == 0) return cudaSuccess;
+    aggregate_apply_kernel<PLANES><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s) {
+    (void)sm_count;
     const uint32_t n = p.n_workers;       // planes = bit length of N
-    if (n < 2) return launch<1>(p, sm_count, s);
-    if (n < 4) return launch<2>(p, sm_count, s);
-    if (n < 8) return launch<3>(p, sm_count, s);
-    if (n < 16) return launch<4>(p, sm_count, s);
-    if (n < 32) return launch<5>(p, sm_count, s);
-    if (n < 64) return launch<6>(p, sm_count, s);
-    if (n < 128) return launch<7>(p, sm_count, s);
-    return launch<8>(p, sm_count, s);
+    if (n < 2) return launch<1>(p, s);
+    if (n < 4) return launch<2>(p, s);
+    if (n < 8) return launch<3>(p, s);
+    if (n < 16) return launch<4>(p, s);
+    if (n < 32) return launch<5>(p, s);
+    if (n < 64) return launch<6>(p, s);
+    if (n < 128) return launch<7>(p, s);
+    return launch<8>(p, s);
 }
 
 }  // namespace dlion

@@ -142,8 +142,13 @@ struct FusedParams {
     int average;
 };
 
-// Host-side launchers (one per .cu file).  grid = 0 asks the launcher to size a
-// persistent grid from the occupancy calculator and sm_count.
+// One thread block per work item, in item order (the kernels still stride, so a
+// count beyond the largest grid is covered too).
+inline unsigned grid_for(unsigned long long n_items) {
+    return n_items > 0x7FFFFFFFull ? 0x7FFFFFFFu : static_cast<unsigned>(n_items);
+}
+
+// Host-side launchers (one per .cu file).
 cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s);
 cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s);
 cudaError_t launch_step_fused(const FusedParams& p, bool bf16, int sm_count, cudaStream_t s);

@@ -126,23 +126,17 @@ step_fused_kernel(const FusedParams p) {
 }
 
 template <bool BF16>
-cudaError_t launch(const FusedParams& p, int sm_count, cudaStream_t s) {
-    int per_sm = 0;
-    cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, step_fused_kernel<BF16>,
-                                                                  kThreads, 0);
-    if (e != cudaSuccess) return e;
-    if (per_sm < 1) per_sm = 1;
-    unsigned long long grid = static_cast<unsigned long long>(per_sm) * sm_count;
-    if (grid > p.ntiles) grid = p.ntiles;
-    if (grid == 0) return cudaSuccess;
-    step_fused_kernel<BF16><<<static_cast<unsigned>(grid), kThreads, 0, s>>>(p);
+cudaError_t launch(const FusedParams& p, cudaStream_t s) {
+    if (p.ntiles == 0) return cudaSuccess;
+    step_fused_kernel<BF16><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 cudaError_t launch_step_fused(const FusedParams& p, bool bf16, int sm_count, cudaStream_t s) {
-    return bf16 ? launch<true>(p, sm_count, s) : launch<false>(p, sm_count, s);
+    (void)sm_count;
+    return bf16 ? launch<true>(p, s) : launch<false>(p, s);
 }
 
 }  // namespace dlion
