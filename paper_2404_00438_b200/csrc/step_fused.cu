@@ -6,7 +6,9 @@
 // written only when the caller asks for it.
 //
 // Same tile and lane mapping as the worker-side kernel (warp = 512 consecutive
-// coordinates, lane l of a chunk = coordinates 4l..4l+3).  HBM traffic per
+// coordinates, lane l of a chunk = coordinates 4l..4l+3).  The
+// worker loop is software-pipelined: worker i+1's loads are issued before worker
+// i is consumed.  HBM traffic per
 // coordinate: N (G + 8) + 8 B, G = gradient bytes (+ N/8 B with the wire buffer):
 // the 2 N/8 B round trip of the two-stage path is gone.
 #include "dlion_common.cuh"
@@ -14,21 +16,113 @@
 namespace dlion {
 namespace {
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;             // 8 warps x 512 coordinates = one tile
 constexpr int kChunksPerWarp = 4;
 
-__device__ __forceinline__ float delta_of(uint32_t count, uint32_t n, uint32_t thr, int average,
-                                          const float* avg_table) {
-    if (average) return avg_table[count];
+template <bool AVG>
+__device__ __forceinline__ float delta_of(uint32_t count, uint32_t thr, const float* avg_table) {
+    if constexpr (AVG) return avg_table[count];
     return count >= thr ? 1.0f : -1.0f;
 }
 
 template <bool BF16>
-__global__ void __launch_bounds__(kThreads)
+struct RawGrad4 { float4 v; };            // four gradients as stored
+template <>
+struct RawGrad4<true> { uint2 v; };
+
+template <bool BF16>
+struct WorkerRegs {                       // one worker's gradients and momenta of my coordinates
+    RawGrad4<BF16> g[kChunksPerWarp];
+    float4 m[kChunksPerWarp];
+    __device__ __forceinline__ void load(const FusedParams& p, unsigned long long at) {
+#pragma unroll
+        for (int u = 0; u < kChunksPerWarp; ++u) {
+            if constexpr (BF16) {
+                g[u].v = __ldcs(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.g) + at + u * kChunk));
+            } else {
+                g[u].v = __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(p.g) + at + u * kChunk));
+            }
+            m[u] = __ldcs(reinterpret_cast<const float4*>(p.m + at + u * kChunk));
+        }
+    }
+    __device__ __forceinline__ float4 grad(int u) const {
+        if constexpr (BF16) {
+            return make_float4(bf16_lo(g[u].v.x), bf16_hi(g[u].v.x), bf16_lo(g[u].v.y), bf16_hi(g[u].v.y));
+        } else {
+            return g[u].v;
+        }
+    }
+};
+
+// Worker-side update of my coordinates for one worker: momenta stored, votes
+// added to cnt (one byte per coordinate), wire words written if requested.
+template <bool BF16>
+__device__ __forceinline__ void consume(const FusedParams& p, WorkerRegs<BF16>& r, unsigned long long at,
+                                        uint32_t* wire_words, uint32_t lane, uint32_t (&cnt)[kChunksPerWarp]) {
+    uint32_t mine = 0;
+#pragma unroll
+    for (int u = 0; u < kChunksPerWarp; ++u) {
+        const float4 g = r.grad(u);
+        uint32_t nib = lion_coord(g.x, r.m[u].x, p.k);
+        nib |= lion_coord(g.y, r.m[u].y, p.k) << 1;
+        nib |= lion_coord(g.z, r.m[u].z, p.k) << 2;
+        nib |= lion_coord(g.w, r.m[u].w, p.k) << 3;
+        __stcs(reinterpret_cast<float4*>(p.m + at + u * kChunk), r.m[u]);
+        cnt[u] += spread_nibble(nib);
+        if (wire_words != nullptr) {                              // block-uniform
+            const uint32_t w = gather_word(nib, lane);
+            if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
+        }
+    }
+    if (wire_words != nullptr && (lane & 7u) < kChunksPerWarp) {
+        wire_words[4u * (lane & 7u) + (lane >> 3)] = mine;
+    }
+}
+
+// Last tile of a segment: every access guarded, one chunk at a time.
+template <bool BF16, bool AVG>
+__device__ __noinline__ void ragged_tile(const FusedParams& p, const TileRef t, uint32_t in_tile,
+                                         unsigned long long e0, uint32_t lane, uint32_t thr,
+                                         const float* avg_table) {
+    const uint32_t n = p.n_workers;
+    const unsigned long long w_stride = p.d_pad / 32;
+#pragma unroll 1
+    for (int u = 0; u < kChunksPerWarp; ++u) {
+        const uint32_t c0 = in_tile + u * kChunk;
+        if (c0 >= t.valid) break;                           // warp-uniform
+        const uint32_t j0 = c0 + lane * 4;
+        const uint32_t mine_n = j0 >= t.valid ? 0u : (t.valid - j0 >= 4u ? 4u : t.valid - j0);
+        uint32_t c4 = 0;
+        for (uint32_t i = 0; i < n; ++i) {
+            const unsigned long long e = i * p.d_pad + e0 + u * kChunk;
+            uint32_t nib = 0;
+            for (uint32_t q = 0; q < mine_n; ++q) {
+                const float g = load_grad1<BF16>(p.g, e + q);
+                float m = p.m[e + q];
+                nib |= lion_coord(g, m, p.k) << q;
+                p.m[e + q] = m;
+            }
+            c4 += spread_nibble(nib);
+            if (p.packed != nullptr) {
+                const uint32_t w = gather_word(nib, lane);
+                if ((lane & 7u) == 0 && c0 + (lane >> 3) * 32 < t.valid) {
+                    p.packed[i * w_stride + (t.base + c0) / 32 + (lane >> 3)] = w;
+                }
+            }
+        }
+        for (uint32_t q = 0; q < mine_n; ++q) {
+            const unsigned long long e = e0 + u * kChunk + q;
+            p.x[e] = apply_coord(p.x[e], delta_of<AVG>((c4 >> (8 * q)) & 0xFFu, thr, avg_table), p.lr, p.wd);
+        }
+    }
+}
+
+template <bool BF16, bool AVG>
+__global__ void __launch_bounds__(kThreads, 2)
 step_fused_kernel(const FusedParams p) {
     __shared__ float avg_table[256];
     const uint32_t n = p.n_workers;
-    if (p.average) {
+    if constexpr (AVG) {
         for (uint32_t c = threadIdx.x; c <= n; c += kThreads) {
             avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
                                      static_cast<float>(n));
@@ -45,82 +139,40 @@ step_fused_kernel(const FusedParams p) {
         const uint32_t in_tile = warp * (kChunksPerWarp * kChunk);
         if (in_tile >= t.valid) continue;                          // warp-uniform
         const unsigned long long e0 = t.base + in_tile + lane * 4;  // my first coordinate (chunk 0)
-        uint32_t cnt[kChunksPerWarp] = {0, 0, 0, 0};
 
         if (t.valid == kTile) {
+            // ---- full tile: while worker i is consumed, worker i+1 is already in flight
+            uint32_t cnt[kChunksPerWarp];
+#pragma unroll
+            for (int u = 0; u < kChunksPerWarp; ++u) cnt[u] = 0;
             float4 xv[kChunksPerWarp];
 #pragma unroll
             for (int u = 0; u < kChunksPerWarp; ++u) {
                 xv[u] = __ldcs(reinterpret_cast<const float4*>(p.x + e0 + u * kChunk));
             }
-#pragma unroll 2
-            for (uint32_t i = 0; i < n; ++i) {
-                const unsigned long long wb = i * p.d_pad + e0;
-                float4 g[kChunksPerWarp], m[kChunksPerWarp];
-#pragma unroll
-                for (int u = 0; u < kChunksPerWarp; ++u) {
-                    g[u] = load_grad4<BF16>(p.g, wb + u * kChunk);
-                    m[u] = __ldcs(reinterpret_cast<const float4*>(p.m + wb + u * kChunk));
-                }
-                uint32_t mine = 0;
-#pragma unroll
-                for (int u = 0; u < kChunksPerWarp; ++u) {
-                    uint32_t nib = lion_coord(g[u].x, m[u].x, p.k);
-                    nib |= lion_coord(g[u].y, m[u].y, p.k) << 1;
-                    nib |= lion_coord(g[u].z, m[u].z, p.k) << 2;
-                    nib |= lion_coord(g[u].w, m[u].w, p.k) << 3;
-                    __stcs(reinterpret_cast<float4*>(p.m + wb + u * kChunk), m[u]);
-                    cnt[u] += spread_nibble(nib);
-                    if (p.packed != nullptr) {
-                        const uint32_t w = gather_word(nib, lane);
-                        if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
-                    }
-                }
-                if (p.packed != nullptr && (lane & 7u) < kChunksPerWarp) {
-                    p.packed[i * w_stride + (t.base + in_tile) / 32 + 4u * (lane & 7u) + (lane >> 3)] = mine;
-                }
+            uint32_t* wire = p.packed == nullptr ? nullptr : p.packed + (t.base + in_tile) / 32;
+            WorkerRegs<BF16> a, b;
+            a.load(p, e0);
+            uint32_t i = 0;
+            for (; i + 2 <= n; i += 2) {
+                b.load(p, (i + 1) * p.d_pad + e0);
+                consume<BF16>(p, a, i * p.d_pad + e0, wire == nullptr ? nullptr : wire + i * w_stride, lane, cnt);
+                if (i + 2 < n) a.load(p, (i + 2) * p.d_pad + e0);
+                consume<BF16>(p, b, (i + 1) * p.d_pad + e0, wire == nullptr ? nullptr : wire + (i + 1) * w_stride,
+                              lane, cnt);
             }
+            if (i < n) consume<BF16>(p, a, i * p.d_pad + e0, wire == nullptr ? nullptr : wire + i * w_stride, lane, cnt);
 #pragma unroll
             for (int u = 0; u < kChunksPerWarp; ++u) {
                 float4 v = xv[u];
-                v.x = apply_coord(v.x, delta_of(cnt[u] & 0xFFu, n, thr, p.average, avg_table), p.lr, p.wd);
-                v.y = apply_coord(v.y, delta_of((cnt[u] >> 8) & 0xFFu, n, thr, p.average, avg_table), p.lr, p.wd);
-                v.z = apply_coord(v.z, delta_of((cnt[u] >> 16) & 0xFFu, n, thr, p.average, avg_table), p.lr, p.wd);
-                v.w = apply_coord(v.w, delta_of(cnt[u] >> 24, n, thr, p.average, avg_table), p.lr, p.wd);
+                v.x = apply_coord(v.x, delta_of<AVG>(cnt[u] & 0xFFu, thr, avg_table), p.lr, p.wd);
+                v.y = apply_coord(v.y, delta_of<AVG>((cnt[u] >> 8) & 0xFFu, thr, avg_table), p.lr, p.wd);
+                v.z = apply_coord(v.z, delta_of<AVG>((cnt[u] >> 16) & 0xFFu, thr, avg_table), p.lr, p.wd);
+                v.w = apply_coord(v.w, delta_of<AVG>(cnt[u] >> 24, thr, avg_table), p.lr, p.wd);
                 __stcs(reinterpret_cast<float4*>(p.x + e0 + u * kChunk), v);
             }
         } else {
-            // last tile of a segment: guarded, one chunk at a time
-#pragma unroll 1
-            for (int u = 0; u < kChunksPerWarp; ++u) {
-                const uint32_t c0 = in_tile + u * kChunk;
-                if (c0 >= t.valid) break;                           // warp-uniform
-                const uint32_t j0 = c0 + lane * 4;
-                const uint32_t mine_n = j0 >= t.valid ? 0u : (t.valid - j0 >= 4u ? 4u : t.valid - j0);
-                uint32_t c4 = 0;
-                for (uint32_t i = 0; i < n; ++i) {
-                    const unsigned long long e = i * p.d_pad + e0 + u * kChunk;
-                    uint32_t nib = 0;
-                    for (uint32_t q = 0; q < mine_n; ++q) {
-                        const float g = load_grad1<BF16>(p.g, e + q);
-                        float m = p.m[e + q];
-                        nib |= lion_coord(g, m, p.k) << q;
-                        p.m[e + q] = m;
-                    }
-                    c4 += spread_nibble(nib);
-                    if (p.packed != nullptr) {
-                        const uint32_t w = gather_word(nib, lane);
-                        if ((lane & 7u) == 0 && c0 + (lane >> 3) * 32 < t.valid) {
-                            p.packed[i * w_stride + (t.base + c0) / 32 + (lane >> 3)] = w;
-                        }
-                    }
-                }
-                for (uint32_t q = 0; q < mine_n; ++q) {
-                    const unsigned long long e = e0 + u * kChunk + q;
-                    p.x[e] = apply_coord(p.x[e], delta_of((c4 >> (8 * q)) & 0xFFu, n, thr, p.average, avg_table),
-                                         p.lr, p.wd);
-                }
-            }
+            ragged_tile<BF16, AVG>(p, t, in_tile, e0, lane, thr, avg_table);
         }
     }
 }
@@ -128,7 +180,11 @@ step_fused_kernel(const FusedParams p) {
 template <bool BF16>
 cudaError_t launch(const FusedParams& p, cudaStream_t s) {
     if (p.ntiles == 0) return cudaSuccess;
-    step_fused_kernel<BF16><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
+    if (p.average) {
+        step_fused_kernel<BF16, true><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
+    } else {
+        step_fused_kernel<BF16, false><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
+    }
     return cudaGetLastError();
 }
 
