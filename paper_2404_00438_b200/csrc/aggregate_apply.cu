@@ -60,8 +60,11 @@ __device__ __forceinline__ void add8(uint32_t (&pl)[kMaxPlanes], const uint32_t*
 }
 
 // Adds the n workers' words of one word position (col, col + w_stride, ...).
-// Up to 16 loads are issued before the adders run, so one round trip to memory
-// covers N = 16.  live = false reads nothing (the word holds no parameter).
+// Whole groups of 16 workers are fetched with 16 loads issued before the adders
+// run; what is left (fewer than 16) goes in ONE more batch of 8 or 16 guarded
+// loads, slots past the last worker adding zero.  So N <= 16 costs one round trip
+// to memory and every further 16 workers one more.
+// live = false reads nothing at all (the word position holds no parameter).
 template <int PLANES>
 __device__ __forceinline__ void count_votes(uint32_t (&pl)[kMaxPlanes], const uint32_t* __restrict__ col,
                                             unsigned long long w_stride, uint32_t n, bool live) {
@@ -78,22 +81,19 @@ __device__ __forceinline__ void count_votes(uint32_t (&pl)[kMaxPlanes], const ui
             add8<PLANES>(pl, w + 8);
         }
     }
-    if constexpr (PLANES >= 4) {
-        for (; i + 8 <= n; i += 8) {
-            uint32_t w[8];
+    const uint32_t rest = n - i;
+    if (PLANES >= 4 && rest > 8) {
+        uint32_t w[16];
 #pragma unroll
-            for (int q = 0; q < 8; ++q) w[q] = __ldg(col + (i + q) * w_stride);
-            add8<PLANES>(pl, w);
-        }
+        for (int q = 0; q < 16; ++q) w[q] = (i + q < n) ? __ldg(col + (i + q) * w_stride) : 0u;
+        add8<PLANES>(pl, w);
+        add8<PLANES>(pl, w + 8);
+    } else if (rest > 0) {
+        uint32_t w[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) w[q] = (i + q < n) ? __ldg(col + (i + q) * w_stride) : 0u;
+        add8<PLANES>(pl, w);
     }
-    for (; i + 4 <= n; i += 4) {
-        uint32_t w[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) w[q] = __ldg(col + (i + q) * w_stride);
-#pragma unroll
-        for (int q = 0; q < 4; ++q) ripple_add<PLANES, 0>(pl, w[q]);
-    }
-    for (; i < n; ++i) ripple_add<PLANES, 0>(pl, __ldg(col + i * w_stride));
 }
 
 // Bit j set where count_j >= thr (bitwise magnitude comparison, MSB first).
@@ -163,23 +163,29 @@ __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, ui
 // (Averaging, or count_out requested).
 template <int PLANES, bool AVG, bool COUNTS>
 __global__ void __launch_bounds__(kThreads, kMinBlocks)
-aggregate_apply_kernel(const AggParams p) {
-    __shared__ float avg_table[256];      // Delta of Averaging for every count P
+aggregate_apply_kernel(const __grid_constant__ AggParams p) {
+    // Delta of Averaging for every count P, one private copy per warp: it is
+    // filled after the tile's first loads are in flight and needs no block barrier.
+    __shared__ float avg_tables[AVG ? kThreads / 32 : 1][AVG ? 256 : 1];
     const uint32_t n = p.n_workers;
-    if constexpr (AVG) {
-        for (uint32_t c = threadIdx.x; c <= n; c += kThreads) {
-            avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
-                                     static_cast<float>(n));
-        }
-        __syncthreads();
-    }
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t thr = (n + 1u) >> 1;   // 2P >= N  <=>  P >= ceil(N/2)
+    float* avg_table = avg_tables[AVG ? warp : 0];
+    bool have_table = !AVG;
+    auto fill_table = [&]() {
+        for (uint32_t c = lane; c <= n; c += 32) {
+            avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
+                                     static_cast<float>(n));
+        }
+        __syncwarp();
+        have_table = true;
+    };
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
         const TileRef t = find_tile(p.segs, p.nseg, tile);
         if (t.valid != kTile) {
+            if (!have_table) fill_table();
             ragged_tile<PLANES, AVG, COUNTS>(p, t, warp, lane, thr, avg_table);
             continue;
         }
@@ -190,6 +196,7 @@ aggregate_apply_kernel(const AggParams p) {
         float4 xv[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) xv[c] = __ldcs(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
+        if (!have_table) fill_table();
         uint32_t pl[kMaxPlanes];
         count_votes<PLANES>(pl, p.packed + word_idx, p.w_stride, n, true);
         const uint32_t dword = planes_ge<PLANES>(pl, thr);

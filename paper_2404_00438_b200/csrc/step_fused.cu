@@ -119,7 +119,7 @@ __device__ __noinline__ void ragged_tile(const FusedParams& p, const TileRef t, 
 
 template <bool BF16, bool AVG>
 __global__ void __launch_bounds__(kThreads, 2)
-step_fused_kernel(const FusedParams p) {
+step_fused_kernel(const __grid_constant__ FusedParams p) {
     __shared__ float avg_table[256];
     const uint32_t n = p.n_workers;
     if constexpr (AVG) {

@@ -26,6 +26,7 @@ namespace {
 constexpr int kThreads = 256;            // 8 warps x 512 coordinates = one tile
 constexpr int kChunksPerWarp = 4;
 
+// (Parameters are taken by value on purpose: marking them __grid_constant__ measured 6 % slower here.)
 template <bool BF16>
 __global__ void __launch_bounds__(kThreads)
 worker_step_kernel(const WorkerParams p) {
