@@ -193,6 +193,16 @@ int dlion_oracle_aggregate_apply(const dlion_oracle_segment* segs, uint32_t nseg
     return 0;
 }
 
+// Number of bit planes of the server->worker message: 1 for Majority Vote (Delta
+// is binary); for Averaging the integer P in {0..N} takes ceil(log2(N+1)) bits
+// (Section 3.2 "Communication Cost"; the paper rounds this to log N).
+uint32_t dlion_oracle_delta_planes(uint32_t n_workers, int mode) {
+    if (mode == DLION_ORACLE_MAJORITY) return 1;
+    uint32_t bits = 0;
+    while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;
+    return bits;
+}
+
 // Analytic communication volume per step in BITS (Table 1 and Section 3.2
 // "Communication Cost"), for d parameters and N workers.
 //   direction 0: all workers -> server, N * d (one bit per parameter per worker)
@@ -201,10 +211,76 @@ int dlion_oracle_aggregate_apply(const dlion_oracle_segment* segs, uint32_t nseg
 //                bits (the paper rounds this to log N)
 uint64_t dlion_oracle_wire_bits(uint64_t d, uint32_t n_workers, int mode, int direction) {
     if (direction == 0) return static_cast<uint64_t>(n_workers) * d;
-    if (mode == DLION_ORACLE_MAJORITY) return d;
-    uint32_t bits = 0;
-    while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;
-    return d * bits;
+    return d * dlion_oracle_delta_planes(n_workers, mode);
+}
+
+// Server side of Algorithm 1 alone: from the N binary vectors, the message that
+// is broadcast to the workers.
+//   Majority Vote: delta_wire[d_pad/32], bit j = 1 iff Delta_j = +1 (S_j >= 0, R2/R3).
+//   Averaging:     K = ceil(log2(N+1)) planes, plane p at delta_wire + p*(d_pad/32):
+//                  bit j of plane p = bit p of P_j (the integer in {0..N}, R4).
+// Words that hold no parameter are left untouched; padding bits of written words are 0.
+int dlion_oracle_aggregate(const dlion_oracle_segment* segs, uint32_t nseg, uint64_t d_pad,
+                           uint32_t n_workers, int mode, const uint32_t* packed,
+                           uint32_t* delta_wire) {
+    if (!segs || !packed || !delta_wire || d_pad % 32 != 0 || n_workers == 0) return -1;
+    if (mode != DLION_ORACLE_MAJORITY && mode != DLION_ORACLE_AVERAGE) return -1;
+    const uint64_t W = d_pad / 32;
+    const uint32_t K = dlion_oracle_delta_planes(n_workers, mode);
+    for (uint32_t s = 0; s < nseg; ++s) {
+        const uint64_t lo = segs[s].elem_offset;
+        const uint64_t hi = lo + segs[s].numel;
+        if (hi > d_pad || lo % 32 != 0) return -1;
+        for (uint64_t w = lo / 32; w < (hi + 31) / 32; ++w) {
+            for (uint32_t p = 0; p < K; ++p) delta_wire[p * W + w] = 0;
+            for (uint32_t b = 0; b < 32; ++b) {
+                const uint64_t j = w * 32 + b;
+                if (j < lo || j >= hi) continue;
+                uint32_t P = 0;
+                for (uint32_t i = 0; i < n_workers; ++i) P += (packed[i * W + w] >> b) & 1u;
+                if (mode == DLION_ORACLE_MAJORITY) {
+                    if (2 * static_cast<int64_t>(P) - static_cast<int64_t>(n_workers) >= 0) delta_wire[w] |= 1u << b;
+                } else {
+                    for (uint32_t p = 0; p < K; ++p) delta_wire[p * W + w] |= ((P >> p) & 1u) << b;
+                }
+            }
+        }
+    }
+    return 0;
+}
+
+// Worker side, first line of Algorithm 1's loop body: every worker applies the
+// broadcast Delta, x <- x - eps (Delta + lambda x), decoding it from the wire
+// format written by dlion_oracle_aggregate.
+int dlion_oracle_apply_delta(const dlion_oracle_segment* segs, uint32_t nseg, uint64_t d_pad,
+                             uint32_t n_workers, int mode, const uint32_t* delta_wire, float* x,
+                             float lr, float weight_decay) {
+    if (!segs || !delta_wire || !x || d_pad % 32 != 0 || n_workers == 0) return -1;
+    if (mode != DLION_ORACLE_MAJORITY && mode != DLION_ORACLE_AVERAGE) return -1;
+    const uint64_t W = d_pad / 32;
+    const uint32_t K = dlion_oracle_delta_planes(n_workers, mode);
+    const int32_t N = static_cast<int32_t>(n_workers);
+    for (uint32_t s = 0; s < nseg; ++s) {
+        const uint64_t lo = segs[s].elem_offset;
+        const uint64_t hi = lo + segs[s].numel;
+        if (hi > d_pad || lo % 32 != 0) return -1;
+        for (uint64_t j = lo; j < hi; ++j) {
+            float Delta;
+            if (mode == DLION_ORACLE_MAJORITY) {
+                Delta = ((delta_wire[j / 32] >> (j % 32)) & 1u) ? 1.0f : -1.0f;
+            } else {
+                int32_t P = 0;
+                for (uint32_t p = 0; p < K; ++p) P |= static_cast<int32_t>((delta_wire[p * W + j / 32] >> (j % 32)) & 1u) << p;
+                Delta = static_cast<float>(2 * P - N) / static_cast<float>(N);
+            }
+            const float xo = x[j];
+            const float u1 = weight_decay * xo;
+            const float u2 = Delta + u1;
+            const float u3 = lr * u2;
+            x[j] = xo - u3;
+        }
+    }
+    return 0;
 }
 
 // 1 when this build honours the nthreads argument (OpenMP), else 0.

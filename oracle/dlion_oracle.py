@@ -56,6 +56,16 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.dlion_oracle_wire_bits.argtypes = [ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int,
                                            ctypes.c_int]
     lib.dlion_oracle_has_openmp.restype = ctypes.c_int
+    lib.dlion_oracle_delta_planes.restype = ctypes.c_uint32
+    lib.dlion_oracle_delta_planes.argtypes = [ctypes.c_uint32, ctypes.c_int]
+    lib.dlion_oracle_aggregate.restype = ctypes.c_int
+    lib.dlion_oracle_aggregate.argtypes = [
+        ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int,
+        ctypes.c_void_p, ctypes.c_void_p]
+    lib.dlion_oracle_apply_delta.restype = ctypes.c_int
+    lib.dlion_oracle_apply_delta.argtypes = [
+        ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int,
+        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_float]
     return lib
 
 
@@ -133,6 +143,34 @@ def wire_bits(d: int, n_workers: int, mode: int, direction: int,
               lib: Optional[ctypes.CDLL] = None) -> int:
     """Table 1: bits per step, worker->server (0) or server->worker (1)."""
     return int((lib or _get()).dlion_oracle_wire_bits(d, n_workers, mode, direction))
+
+
+def delta_planes(n_workers: int, mode: int, lib: Optional[ctypes.CDLL] = None) -> int:
+    """Bit planes of the server->worker message: 1 (Majority Vote) or ceil(log2(N+1))."""
+    return int((lib or _get()).dlion_oracle_delta_planes(n_workers, mode))
+
+
+def aggregate(segments, d_pad: int, n_workers: int, mode: int, packed: np.ndarray,
+              delta_wire: np.ndarray, lib: Optional[ctypes.CDLL] = None) -> None:
+    """Alg. 1 server side alone: writes the broadcast message (bits, or count bit planes)."""
+    _check(packed, np.uint32, n_workers * d_pad // 32, "packed")
+    _check(delta_wire, np.uint32, delta_planes(n_workers, mode, lib) * d_pad // 32, "delta_wire")
+    rc = (lib or _get()).dlion_oracle_aggregate(_segs(segments), len(segments), d_pad, n_workers, mode,
+                                                _ptr(packed), _ptr(delta_wire))
+    if rc != 0:
+        raise ValueError("dlion_oracle_aggregate rejected its arguments")
+
+
+def apply_delta(segments, d_pad: int, n_workers: int, mode: int, delta_wire: np.ndarray,
+                x: np.ndarray, lr: float, weight_decay: float,
+                lib: Optional[ctypes.CDLL] = None) -> None:
+    """Alg. 1 worker side, first line: x <- x - eps (Delta + lambda x) from the wire format."""
+    _check(delta_wire, np.uint32, delta_planes(n_workers, mode, lib) * d_pad // 32, "delta_wire")
+    _check(x, np.float32, d_pad, "x")
+    rc = (lib or _get()).dlion_oracle_apply_delta(_segs(segments), len(segments), d_pad, n_workers, mode,
+                                                  _ptr(delta_wire), _ptr(x), lr, weight_decay)
+    if rc != 0:
+        raise ValueError("dlion_oracle_apply_delta rejected its arguments")
 
 
 def has_openmp() -> bool:

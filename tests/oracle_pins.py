@@ -339,7 +339,56 @@ def check_wire_bits(lib):
     assert 32 * d // orc.wire_bits(d, 1, MAJ, 1, lib=lib) == 32
 
 
+# ---------------------------------------------------------------- server->worker wire format
+def check_delta_wire_roundtrip(lib):
+    """aggregate() writes Delta as broadcast (bits, or ceil(log2(N+1)) count bit planes: Section 3.2
+    "Communication Cost"); apply_delta() decodes it.  Planes must decode to the brute-force counts,
+    and the two halves together must equal the one-call server step."""
+    rng = np.random.default_rng(10)
+    segs = [(0, 70), (128, 1), (256, 33), (384, 64)]
+    d_pad = 512
+    W = d_pad // 32
+    valid = np.zeros(d_pad, bool)
+    for o, n in segs:
+        valid[o:o + n] = True
+    d = int(valid.sum())
+    for N in (1, 2, 3, 4, 7, 8, 16, 33, 255):
+        bits = (rng.random((N, d_pad)) < rng.random(d_pad)[None, :]) & valid[None, :]
+        packed = np.packbits(bits, axis=1, bitorder="little").view(np.uint32).reshape(N, -1).copy()
+        P = bits.sum(axis=0).astype(np.int64)
+        for mode in (MAJ, AVG):
+            K = orc.delta_planes(N, mode, lib=lib)
+            assert K == (1 if mode == MAJ else int(np.ceil(np.log2(N + 1))))
+            assert K * d == orc.wire_bits(d, N, mode, 1, lib=lib)
+            wire = np.full(K * W, 0xFFFFFFFF, np.uint32)          # garbage: must be overwritten or left alone
+            orc.aggregate(segs, d_pad, N, mode, packed, wire, lib=lib)
+            planes = unpack(wire.reshape(K, W), d_pad).astype(np.int64)
+            if mode == MAJ:
+                assert np.array_equal(planes[0][valid], (2 * P >= N)[valid].astype(np.int64))
+            else:
+                decoded = sum(planes[p] << p for p in range(K))
+                assert np.array_equal(decoded[valid], P[valid])
+            touched = np.zeros(W, bool)
+            for o, n in segs:
+                touched[o // 32:(o + n + 31) // 32] = True
+            assert np.all(wire.reshape(K, W)[:, ~touched] == 0xFFFFFFFF)
+            pad_in_touched = ~valid & np.repeat(touched, 32)
+            assert not planes[:, pad_in_touched].any()
+            x0 = f32(rng.standard_normal(d_pad))
+            lr, wd = 0.125, 0.5
+            xa, xb = x0.copy(), x0.copy()
+            orc.apply_delta(segs, d_pad, N, mode, wire, xa, lr, wd, lib=lib)
+            orc.aggregate_apply(segs, d_pad, N, mode, packed, xb, lr, wd, lib=lib)
+            assert np.array_equal(xa, xb)
+            S = 2 * P - N
+            Delta = S / N if mode == AVG else np.where(S >= 0, 1.0, -1.0)
+            want = x0.astype(np.float64) - lr * (Delta + wd * x0.astype(np.float64))
+            assert np.abs(xa[valid] - want[valid]).max() <= 2 * np.spacing(np.float32(4.0))
+            assert np.array_equal(xa[~valid], x0[~valid])
+
+
 ALL_CHECKS = [check_hand_case, check_sign_of_zero_and_tie, check_delta_is_sign_of_blend,
               check_single_worker_is_lion, check_identical_workers, check_beta_zero_is_signsgd,
               check_equal_betas_is_signum, check_counts_bruteforce, check_x_closed_form,
-              check_phase_one_contraction, check_padding_untouched, check_wire_bits]
+              check_phase_one_contraction, check_padding_untouched, check_wire_bits,
+              check_delta_wire_roundtrip]

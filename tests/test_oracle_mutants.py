@@ -30,6 +30,15 @@ MUTANTS = {
                                   "P += static_cast<int32_t>((packed[static_cast<size_t>(0) * W"),
     "padding_written": ("if (j < lo || j >= hi) continue;            // padding bit stays 0",
                         "if (j >= d_pad) continue;"),
+    "wire_planes_reversed": ("delta_wire[p * W + w] |= ((P >> p) & 1u) << b;",
+                             "delta_wire[p * W + w] |= ((P >> (K - 1 - p)) & 1u) << b;"),
+    "wire_majority_bit_inverted": ("Delta = ((delta_wire[j / 32] >> (j % 32)) & 1u) ? 1.0f : -1.0f;",
+                                   "Delta = ((delta_wire[j / 32] >> (j % 32)) & 1u) ? -1.0f : 1.0f;"),
+    "wire_decode_without_doubling": ("Delta = static_cast<float>(2 * P - N) / static_cast<float>(N);",
+                                     "Delta = static_cast<float>(P - N) / static_cast<float>(N);"),
+    "wire_apply_sign": ("x[j] = xo - u3;", "x[j] = xo + u3;"),
+    "wire_tie_negative": ("static_cast<int64_t>(n_workers) >= 0) delta_wire[w] |= 1u << b;",
+                          "static_cast<int64_t>(n_workers) > 0) delta_wire[w] |= 1u << b;"),
     "average_down_bits_floor_log": ("while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;",
                                     "while ((2ull << bits) <= static_cast<uint64_t>(n_workers)) ++bits;"),
 }
