@@ -18,9 +18,7 @@ import hashlib
 import json
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
 import time
 
 import numpy as np
@@ -60,53 +58,70 @@ def measured_peak():
 
 
 class ClockSampler:
-    """nvidia-smi polled every 200 ms while the timed region runs (read-only)."""
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Read-only NVML polling (every 20 ms, in a thread) of SM clock, power and clock-event
+    reasons; the summary covers the samples taken inside [window_start, window_end]."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
 
-    def __init__(self, gpu_index: int):
-        self.gpu, self.proc, self.path = gpu_index, None, None
+    def __init__(self, cuda_index: int):
+        self.samples, self.thread, self.stop_flag, self.handle, self.nv = [], None, False, None, None
+        self.t0 = self.t1 = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(cuda_index).uuid)
+            try:
+                self.handle = pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid) if not uuid.startswith("GPU-") else uuid)
+            except Exception:
+                self.handle = pynvml.nvmlDeviceGetHandleByIndex(cuda_index)
+            self.nv = pynvml
+        except Exception:
+            self.nv = None
+
+    def _loop(self):
+        nv, h = self.nv, self.handle
+        while not self.stop_flag:
+            try:
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                self.samples.append((time.time(), nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM),
+                                     nv.nvmlDeviceGetPowerUsage(h) / 1000.0, int(reasons)))
+            except Exception:
+                pass
+            time.sleep(0.02)
 
     def start(self):
-        try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "200"],
-                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
-        except Exception:
-            self.proc = None
+        if self.nv is None:
+            return
+        import threading
+        self.thread = threading.Thread(target=self._loop, daemon=True)
+        self.thread.start()
+
+    def window_start(self):
+        self.t0 = time.time()
+
+    def window_end(self):
+        self.t1 = time.time()
 
     def stop(self):
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
+        if self.nv is None or self.thread is None:
+            out["note"] = "NVML unavailable"
             return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, reasons, smax, power = [], set(), None, []
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for line in open(self.path):
-            f = [v.strip() for v in line.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1]))
-                smax = float(f[2])
-                power.append(float(f[3]))
-            except ValueError:
-                continue
-            for name, v in zip(names, f[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        os.unlink(self.path)
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=smax, reasons=sorted(reasons),
-                       samples=len(sm), power_w_max=max(power))
+        self.stop_flag = True
+        self.thread.join(timeout=2)
+        inside = [s for s in self.samples if self.t0 is not None and self.t0 <= s[0] <= (self.t1 or 1e30)]
+        use, scope = (inside, "timed region") if len(inside) >= 3 else (self.samples, "whole measured phase")
+        if use:
+            bits = 0
+            for s in use:
+                bits |= s[3]
+            out.update(sm_mhz=statistics.median(s[1] for s in use),
+                       sm_max_mhz=self.nv.nvmlDeviceGetMaxClockInfo(self.handle, self.nv.NVML_CLOCK_SM),
+                       reasons=sorted(name for bit, name in self.REASONS.items() if bits & bit),
+                       samples=len(use), power_w_max=max(s[2] for s in use), scope=scope)
         return out
 
 
@@ -241,15 +256,30 @@ def run_ours(args):
         step()
     barrier()
 
-    # ---- timed region: K steps, fresh gradients generated between steps (untimed)
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    launches0 = ctx.launch_count()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+
+    # ---- secondary leg: K steps with fresh seeded gradients generated between steps
+    # (generation untimed; each step bracketed by its own events)
+    fresh = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(args.steps)]
     for t in range(args.steps):
         inputs.fill_grads(w, args.warmup + t, g)
         barrier()
+        fresh[t][0].record(stream)
+        step()
+        fresh[t][1].record(stream)
+    barrier()
+    fresh_ms = sum(e[0].elapsed_time(e[1]) for e in fresh) / args.steps
+
+    # ---- timed region: exactly K steps back to back inside one barrier/synchronize
+    # bracket, on the gradients of the last generated step; events between the
+    # kernels give the per-kernel durations
+    launches0 = ctx.launch_count()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    barrier()
+    sampler.window_start()
+    for t in range(args.steps):
         ev[t][0].record(stream)
         if args.path == "fused":
             ctx.step_fused(g, m, x, None)
@@ -260,20 +290,11 @@ def run_ours(args):
             ctx.aggregate_apply(packed, x)
         ev[t][2].record(stream)
     barrier()
+    sampler.window_end()
     launches = ctx.launch_count() - launches0
     k1_ms = [e[0].elapsed_time(e[1]) for e in ev]
     k2_ms = [e[1].elapsed_time(e[2]) for e in ev]
-    total_ms = sum(e[0].elapsed_time(e[2]) for e in ev)
-
-    # ---- the same K steps back to back on the last gradients (sustained clocks)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
-    b2b_ms = e0.elapsed_time(e1) / args.steps
+    total_ms = ev[0][0].elapsed_time(ev[-1][2])
     clocks = sampler.stop() if rank == 0 else None
 
     t_all = torch.tensor([total_ms], dtype=torch.float64, device=dev)
@@ -324,9 +345,9 @@ def run_ours(args):
                        "mode": "average" if mode else "majority", "path": args.path,
                        "l2": "inputs larger than L2 (no flush needed)" if N * D * (w.grad_bytes + 4) > 4 * 126e6
                              else "working set comparable to L2: latency-bound case",
-                       "grads_per_step": "fresh seeded gradients generated between timed steps, untimed",
+                       "timed_region": "K steps back to back in one bracket, on the last generated gradients",
                        "per_rank": "each rank steps its own full-size coordinate slab; no collective"},
-            "ms_per_step_back_to_back": b2b_ms,
+            "ms_per_step_fresh_grads": fresh_ms,
             "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches, "clocks": clocks,
             "wire_bytes_per_step": {"up_all_workers": up, "down_per_worker": down,

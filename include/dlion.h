@@ -114,6 +114,33 @@ dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float
                                    uint32_t* delta_bits_out, uint8_t* count_out,
                                    void* cuda_stream);
 
+/* Server side of Algorithm 1 ALONE (no parameter update): from the N binary
+ * vectors, the message the server broadcasts (Section 3.2, "Communication
+ * Cost"; Table 1, server->worker column).
+ *   packed      in   [N][d_pad/32]
+ *   delta_wire  out  dlion_delta_planes(ctx) planes of d_pad/32 words, plane p at
+ *               delta_wire + p*(d_pad/32).  Majority Vote: one plane, bit = 1 iff
+ *               Delta = +1.  Averaging: K = ceil(log2(N+1)) planes, bit j of plane
+ *               p = bit p of P_j, the integer in {0..N} the paper describes; K*d
+ *               bits in all.  Words that hold no parameter are not written;
+ *               padding bits of written words are 0. */
+dlion_status dlion_aggregate(dlion_ctx* ctx, const uint32_t* packed, uint32_t* delta_wire,
+                             void* cuda_stream);
+
+/* Worker side, first line of the loop body of Algorithm 1: every worker applies
+ * the broadcast update, x <- x - eps (Delta + lambda x), with Delta decoded from
+ * the message written by dlion_aggregate (Averaging: Delta = (2P-N)/N).
+ * dlion_aggregate + dlion_apply_delta give exactly what dlion_aggregate_apply gives.
+ *   delta_wire  in      as written by dlion_aggregate
+ *   x           in/out  parameters */
+dlion_status dlion_apply_delta(dlion_ctx* ctx, const uint32_t* delta_wire, float* x,
+                               void* cuda_stream);
+
+/* Number of d-bit planes of the server->worker message: 1 for Majority Vote,
+ * ceil(log2(N+1)) for Averaging (the paper's "log(N) bits" per parameter).
+ * 0 for a null context. */
+uint32_t dlion_delta_planes(const dlion_ctx* ctx);
+
 /* The whole of one Algorithm-1 iteration in ONE launch: a thread block holds a
  * tile of coordinates for all N workers, votes in registers and applies x.
  * Same results as dlion_worker_step(-1) followed by dlion_aggregate_apply.

@@ -142,6 +142,20 @@ struct FusedParams {
     int average;
 };
 
+struct WireParams {                  // server-only aggregate / worker-side apply
+    const uint32_t* packed;          // aggregate: the N binary vectors
+    uint32_t* wire_out;              // aggregate: the broadcast message
+    const uint32_t* wire_in;         // apply: the broadcast message
+    float* x;                        // apply: parameters
+    const SegDev* segs;
+    uint32_t nseg;
+    uint32_t n_workers;
+    unsigned long long ntiles;
+    unsigned long long w_stride;     // words per binary vector / per plane (d_pad / 32)
+    float lr, wd;
+    int average;
+};
+
 // One thread block per work item, in item order (the kernels still stride, so a
 // count beyond the largest grid is covered too).
 inline unsigned grid_for(unsigned long long n_items) {
@@ -152,5 +166,7 @@ inline unsigned grid_for(unsigned long long n_items) {
 cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s);
 cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s);
 cudaError_t launch_step_fused(const FusedParams& p, bool bf16, int sm_count, cudaStream_t s);
+cudaError_t launch_wire(const WireParams& p, bool apply, cudaStream_t s);
+uint32_t planes_for(uint32_t n_workers);   // ceil(log2(N+1))
 
 }  // namespace dlion

@@ -77,6 +77,53 @@ dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, float* m, f
     return DLION_OK;
 }
 
+uint32_t dlion_delta_planes(const dlion_ctx* ctx) {
+    if (ctx == nullptr) return 0;
+    return ctx->mode == DLION_AVERAGE ? dlion::planes_for(ctx->n_workers) : 1u;
+}
+
+dlion_status dlion_aggregate(dlion_ctx* ctx, const uint32_t* packed, uint32_t* delta_wire, void* cuda_stream) {
+    if (ctx == nullptr || packed == nullptr || delta_wire == nullptr) return DLION_EINVAL;
+    if (!aligned16(packed) || !aligned16(delta_wire)) return DLION_EALIGN;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
+    if (dev != ctx->device) return DLION_ESTATE;
+    dlion::WireParams p{};
+    p.packed = packed;
+    p.wire_out = delta_wire;
+    p.segs = ctx->segs_dev;
+    p.nseg = ctx->nseg;
+    p.n_workers = ctx->n_workers;
+    p.ntiles = ctx->ntiles;
+    p.w_stride = ctx->d_pad / 32;
+    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    if (dlion::launch_wire(p, false, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+dlion_status dlion_apply_delta(dlion_ctx* ctx, const uint32_t* delta_wire, float* x, void* cuda_stream) {
+    if (ctx == nullptr || delta_wire == nullptr || x == nullptr) return DLION_EINVAL;
+    if (!aligned16(delta_wire) || !aligned16(x)) return DLION_EALIGN;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
+    if (dev != ctx->device) return DLION_ESTATE;
+    dlion::WireParams p{};
+    p.wire_in = delta_wire;
+    p.x = x;
+    p.segs = ctx->segs_dev;
+    p.nseg = ctx->nseg;
+    p.n_workers = ctx->n_workers;
+    p.ntiles = ctx->ntiles;
+    p.w_stride = ctx->d_pad / 32;
+    p.lr = ctx->lr;
+    p.wd = ctx->wd;
+    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    if (dlion::launch_wire(p, true, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
 uint64_t dlion_wire_bytes(const dlion_ctx* ctx, int direction) {
     if (ctx == nullptr) return 0;
     const uint64_t d = ctx->d;

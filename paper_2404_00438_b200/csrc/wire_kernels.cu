@@ -1,0 +1,147 @@
+// The two halves of the server round trip of Algorithm 1 (arXiv 2404.00438) as
+// separate kernels, for deployments where the vote and the update run in
+// different places:
+//
+//   aggregate_kernel    server side: from the N binary vectors, the message that
+//                       is broadcast.  Majority Vote: d bits (bit = 1 iff
+//                       Delta = +1).  Averaging: the integer P in {0..N} per
+//                       coordinate (Section 3.2, "Communication Cost") as
+//                       K = ceil(log2(N+1)) bit planes of d bits each, plane p
+//                       holding bit p of every P -- exactly the K*d bits of
+//                       Table 1, and exactly the counters the vote already keeps.
+//   apply_delta_kernel  worker side, first line of the loop body of Algorithm 1:
+//                       x <- x - eps (Delta + lambda x), Delta decoded from that
+//                       message.
+//
+// Run one after the other they give what aggregate_apply_kernel gives in one pass.
+// Traffic per coordinate: aggregate N/8 + K/8 B; apply 8 + K/8 B.
+#include "vote_planes.cuh"
+
+namespace dlion {
+namespace {
+
+constexpr int kThreads = 128;             // 4 warps x 1024 coordinates = one tile
+
+template <int PLANES, bool AVG>
+__global__ void __launch_bounds__(kThreads)
+aggregate_kernel(const __grid_constant__ WireParams p) {
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp = threadIdx.x >> 5;
+    const uint32_t thr = (p.n_workers + 1u) >> 1;
+    for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
+        const TileRef t = find_tile(p.segs, p.nseg, tile);
+        const uint32_t my0 = warp * kWarpSpan + lane * 32;          // first coordinate of my word
+        if (my0 >= t.valid) continue;                               // my word holds no parameter
+        const uint32_t nbits = t.valid - my0 >= 32u ? 32u : t.valid - my0;
+        const uint32_t vmask = nbits == 32u ? kFull : ((1u << nbits) - 1u);
+        const unsigned long long word_idx = (t.base + my0) / 32;
+        uint32_t pl[kMaxPlanes];
+        count_votes<PLANES>(pl, p.packed + word_idx, p.w_stride, p.n_workers, true);
+        if constexpr (AVG) {
+#pragma unroll
+            for (int q = 0; q < PLANES; ++q) p.wire_out[q * p.w_stride + word_idx] = pl[q] & vmask;
+        } else {
+            p.wire_out[word_idx] = planes_ge<PLANES>(pl, thr) & vmask;
+        }
+    }
+}
+
+template <int PLANES, bool AVG>
+__global__ void __launch_bounds__(kThreads, 6)
+apply_delta_kernel(const __grid_constant__ WireParams p) {
+    __shared__ float avg_tables[AVG ? kThreads / 32 : 1][AVG ? 256 : 1];
+    const uint32_t n = p.n_workers;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp = threadIdx.x >> 5;
+    float* avg_table = avg_tables[AVG ? warp : 0];
+    bool have_table = !AVG;
+
+    for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
+        const TileRef t = find_tile(p.segs, p.nseg, tile);
+        const uint32_t w0 = warp * kWarpSpan;
+        if (w0 >= t.valid) continue;                                // warp-uniform
+        const bool full = w0 + kWarpSpan <= t.valid;
+        const unsigned long long xe = t.base + w0 + lane * 4;
+        const unsigned long long word_idx = (t.base + w0) / 32 + lane;
+        const bool live = w0 + lane * 32 < t.valid;                 // my word holds a parameter
+
+        float4 xv[8];
+        if (full) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) xv[c] = __ldcs(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
+        }
+        uint32_t pl[kMaxPlanes];
+        uint32_t dword = 0;
+        if constexpr (AVG) {
+#pragma unroll
+            for (int q = 0; q < PLANES; ++q) pl[q] = live ? __ldg(p.wire_in + q * p.w_stride + word_idx) : 0u;
+        } else {
+            dword = live ? __ldg(p.wire_in + word_idx) : 0u;
+        }
+        if (!have_table) {
+            for (uint32_t c = lane; c <= n; c += 32) {
+                avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
+                                         static_cast<float>(n));
+            }
+            __syncwarp();
+            have_table = true;
+        }
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+            uint32_t dn, cnt4;
+            my_votes<PLANES, AVG>(pl, dword, c, lane, dn, cnt4);
+            const uint32_t j0 = w0 + c * kChunk + lane * 4;
+            if (j0 >= t.valid) continue;                            // after the shuffles: all lanes took part
+            const unsigned long long e = xe + c * kChunk;
+            if (full) {
+                float4 v = xv[c];
+                v.x = apply_coord(v.x, delta_value<AVG>(dn, cnt4, 0, avg_table), p.lr, p.wd);
+                v.y = apply_coord(v.y, delta_value<AVG>(dn, cnt4, 1, avg_table), p.lr, p.wd);
+                v.z = apply_coord(v.z, delta_value<AVG>(dn, cnt4, 2, avg_table), p.lr, p.wd);
+                v.w = apply_coord(v.w, delta_value<AVG>(dn, cnt4, 3, avg_table), p.lr, p.wd);
+                __stcs(reinterpret_cast<float4*>(p.x + e), v);
+            } else {
+                for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
+                    p.x[e + q] = apply_coord(p.x[e + q], delta_value<AVG>(dn, cnt4, q, avg_table), p.lr, p.wd);
+                }
+            }
+        }
+    }
+}
+
+template <int PLANES>
+cudaError_t launch(const WireParams& p, bool apply, cudaStream_t s) {
+    if (p.ntiles == 0) return cudaSuccess;
+    const unsigned grid = grid_for(p.ntiles);
+    if (apply) {
+        if (p.average) apply_delta_kernel<PLANES, true><<<grid, kThreads, 0, s>>>(p);
+        else apply_delta_kernel<1, false><<<grid, kThreads, 0, s>>>(p);
+    } else {
+        if (p.average) aggregate_kernel<PLANES, true><<<grid, kThreads, 0, s>>>(p);
+        else aggregate_kernel<PLANES, false><<<grid, kThreads, 0, s>>>(p);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+uint32_t planes_for(uint32_t n_workers) {      // bit length of N = ceil(log2(N+1))
+    uint32_t k = 0;
+    while ((1u << k) < n_workers + 1u) ++k;
+    return k;
+}
+
+cudaError_t launch_wire(const WireParams& p, bool apply, cudaStream_t s) {
+    switch (planes_for(p.n_workers)) {
+        case 1: return launch<1>(p, apply, s);
+        case 2: return launch<2>(p, apply, s);
+        case 3: return launch<3>(p, apply, s);
+        case 4: return launch<4>(p, apply, s);
+        case 5: return launch<5>(p, apply, s);
+        case 6: return launch<6>(p, apply, s);
+        case 7: return launch<7>(p, apply, s);
+        default: return launch<8>(p, apply, s);
+    }
+}
+
+}  // namespace dlion

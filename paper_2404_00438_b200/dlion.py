@@ -22,7 +22,8 @@ MAX_WORKERS = 255
 OK, EINVAL, EALIGN, ENOMEM, ECUDA, ESTATE = range(6)
 
 EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_worker_step",
-           "dlion_aggregate_apply", "dlion_step_fused", "dlion_step_host", "dlion_step_static",
+           "dlion_aggregate_apply", "dlion_aggregate", "dlion_apply_delta", "dlion_delta_planes",
+           "dlion_step_fused", "dlion_step_host", "dlion_step_static",
            "dlion_wire_bytes",
            "dlion_launch_count", "dlion_status_str", "dlion_destroy")
 
@@ -56,6 +57,12 @@ def _load() -> ctypes.CDLL:
     lib.dlion_worker_step.restype = i32
     lib.dlion_aggregate_apply.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.dlion_aggregate_apply.restype = i32
+    lib.dlion_aggregate.argtypes = [vp, vp, vp, vp]
+    lib.dlion_aggregate.restype = i32
+    lib.dlion_apply_delta.argtypes = [vp, vp, vp, vp]
+    lib.dlion_apply_delta.restype = i32
+    lib.dlion_delta_planes.argtypes = [vp]
+    lib.dlion_delta_planes.restype = u32
     lib.dlion_step_fused.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.dlion_step_fused.restype = i32
     lib.dlion_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
@@ -152,6 +159,17 @@ class Dlion:
                         count_out: Optional[torch.Tensor] = None) -> None:
         self._check(_lib.dlion_aggregate_apply(self._ctx, _ptr(packed), _ptr(x), _ptr(delta_bits_out),
                                                _ptr(count_out), _stream()), "dlion_aggregate_apply")
+
+    def aggregate(self, packed: torch.Tensor, delta_wire: torch.Tensor) -> None:
+        self._check(_lib.dlion_aggregate(self._ctx, _ptr(packed), _ptr(delta_wire), _stream()),
+                    "dlion_aggregate")
+
+    def apply_delta(self, delta_wire: torch.Tensor, x: torch.Tensor) -> None:
+        self._check(_lib.dlion_apply_delta(self._ctx, _ptr(delta_wire), _ptr(x), _stream()),
+                    "dlion_apply_delta")
+
+    def delta_planes(self) -> int:
+        return int(_lib.dlion_delta_planes(self._ctx))
 
     def step_fused(self, grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor,
                    packed_out: Optional[torch.Tensor] = None) -> None:

@@ -172,3 +172,41 @@ def test_step_host_matches_oracle(dl, mode):
         want = ora.count[mode] if mode == AVG else ora.dbits[mode].view(np.uint8)
         gp.compare("wire", host_wire.numpy(), want, True)
     ctx.destroy()
+
+
+# ---------------------------------------------------------------- server-only aggregate + worker-side apply
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 7, 8, 16, 33, 64, 255])
+@pytest.mark.parametrize("mode", [MAJ, AVG])
+def test_aggregate_then_apply_delta(dl, n, mode):
+    from oracle import dlion_oracle as orc
+    w = inputs.custom(RAGGED + [3 * 4096 + 5], n, mode, "f32", lr=1e-2, weight_decay=0.5)
+    dev = torch.device("cuda:0")
+    D, W = w.d_pad, w.d_pad // 32
+    rng = np.random.default_rng(n * 2 + mode)
+    valid = np.zeros(D, bool)
+    for off, cnt in w.segments:
+        valid[off:off + cnt] = True
+    bits = (rng.random((n, D)) < rng.random(D)[None, :]) & valid[None, :]
+    packed_np = np.packbits(bits, axis=1, bitorder="little").view(np.uint32).reshape(n, -1).copy()
+    x0 = inputs.fill_x0(w, torch.empty(D))
+    ctx = gp.make_ctx(dl, w)
+    K = ctx.delta_planes()
+    assert K == orc.delta_planes(n, mode)
+    # oracle
+    wire_ref = np.zeros(K * W, np.uint32)
+    orc.aggregate(w.segments, D, n, mode, packed_np, wire_ref)
+    x_ref = x0.numpy().copy()
+    orc.apply_delta(w.segments, D, n, mode, wire_ref, x_ref, w.lr, w.weight_decay)
+    # CUDA library
+    packed = torch.from_numpy(packed_np.view(np.int32)).to(dev)
+    wire = torch.zeros(K * W, dtype=torch.int32, device=dev)
+    x = x0.to(dev)
+    x_one = x0.to(dev)
+    ctx.aggregate(packed, wire)
+    ctx.apply_delta(wire, x)
+    ctx.aggregate_apply(packed, x_one)
+    torch.cuda.synchronize()
+    gp.compare("delta wire", wire.cpu().numpy().view(np.uint32), wire_ref, True)
+    gp.compare("x after apply_delta", x.cpu().numpy(), x_ref, True)
+    assert torch.equal(x, x_one)
+    ctx.destroy()
