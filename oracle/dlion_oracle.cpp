@@ -63,6 +63,7 @@ struct dlion_oracle_segment {
 
 enum { DLION_ORACLE_MAJORITY = 0, DLION_ORACLE_AVERAGE = 1 };
 enum { DLION_ORACLE_GRAD_F32 = 0, DLION_ORACLE_GRAD_BF16 = 1 };
+enum { DLION_ORACLE_STATE_F32 = 0, DLION_ORACLE_STATE_BF16 = 1 };
 
 }  // extern "C"
 
@@ -82,6 +83,28 @@ inline float load_grad(const void* g, int gdtype, size_t idx) {
     return static_cast<const float*>(g)[idx];
 }
 
+// Momentum kept in bf16 (optional): widened exactly on load; on store the binary32
+// result is rounded to the nearest bf16, ties to the even mantissa (IEEE
+// round-to-nearest-even on the upper 16 bits).  NaN stays NaN (quiet bit set).
+inline uint16_t round_to_bf16(float f) {
+    uint32_t u;
+    std::memcpy(&u, &f, sizeof u);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return static_cast<uint16_t>((u >> 16) | 0x0040u);
+    const uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + lsb;
+    return static_cast<uint16_t>(u >> 16);
+}
+
+inline float load_state(const void* m, int mdtype, size_t idx) {
+    if (mdtype == DLION_ORACLE_STATE_BF16) return widen_bf16(static_cast<const uint16_t*>(m)[idx]);
+    return static_cast<const float*>(m)[idx];
+}
+
+inline void store_state(void* m, int mdtype, size_t idx, float v) {
+    if (mdtype == DLION_ORACLE_STATE_BF16) static_cast<uint16_t*>(m)[idx] = round_to_bf16(v);
+    else static_cast<float*>(m)[idx] = v;
+}
+
 // R2: two-valued sign as a bit.
 inline uint32_t sign_bit(float v) { return (v >= 0.0f) ? 1u : 0u; }
 
@@ -96,14 +119,15 @@ extern "C" {
 //   packed  [N][d_pad/32] delta_{i,t}, one bit per coordinate     (written:
 //           words that hold at least one parameter; others untouched)
 // Returns 0, or -1 on a malformed argument.
-int dlion_oracle_worker_step(const dlion_oracle_segment* segs, uint32_t nseg,
-                             uint64_t d_pad, uint32_t n_workers, int gdtype,
-                             const void* g, float* m, uint32_t* packed,
-                             float beta1, float beta2, int nthreads) {
-    if (!segs || !g || !m || !packed || d_pad % 32 != 0 || n_workers == 0) return -1;
+// General form.  Algorithm 1 lets every worker set its own beta1, beta2 (footnote
+// to its inputs): beta1s[i], beta2s[i] are worker i's.  mdtype selects fp32 or
+// bf16 storage of the momentum (arithmetic is binary32 either way).
+int dlion_oracle_worker_step_ex(const dlion_oracle_segment* segs, uint32_t nseg,
+                                uint64_t d_pad, uint32_t n_workers, int gdtype, int mdtype,
+                                const void* g, void* m, uint32_t* packed,
+                                const float* beta1s, const float* beta2s, int nthreads) {
+    if (!segs || !g || !m || !packed || !beta1s || !beta2s || d_pad % 32 != 0 || n_workers == 0) return -1;
     const uint64_t W = d_pad / 32;
-    const float om1 = 1.0f - beta1;   // R1: (1-beta) in binary32
-    const float om2 = 1.0f - beta2;
     (void)nthreads;
     for (uint32_t s = 0; s < nseg; ++s) {
         const uint64_t lo = segs[s].elem_offset;
@@ -120,21 +144,40 @@ int dlion_oracle_worker_step(const dlion_oracle_segment* segs, uint32_t nseg,
                     const uint64_t j = static_cast<uint64_t>(w) * 32 + b;
                     if (j < lo || j >= hi) continue;            // padding bit stays 0
                     const size_t idx = static_cast<size_t>(i) * d_pad + j;
+                    const float beta1 = beta1s[i], beta2 = beta2s[i];
+                    const float om1 = 1.0f - beta1;             // R1: (1-beta) in binary32
+                    const float om2 = 1.0f - beta2;
                     const float gf = load_grad(g, gdtype, idx);
-                    const float mo = m[idx];                    // R5: old momentum
+                    const float mo = load_state(m, mdtype, idx);  // R5: old momentum
                     const float a1 = beta1 * mo;
                     const float b1 = om1 * gf;
                     const float c = a1 + b1;                    // Alg. 1, delta line
                     word |= sign_bit(c) << b;
                     const float a2 = beta2 * mo;
                     const float b2 = om2 * gf;
-                    m[idx] = a2 + b2;                           // Alg. 1, momentum line
+                    store_state(m, mdtype, idx, a2 + b2);       // Alg. 1, momentum line
                 }
                 packed[static_cast<size_t>(i) * W + static_cast<size_t>(w)] = word;
             }
         }
     }
     return 0;
+}
+
+// The common case: one (beta1, beta2) for all workers, fp32 momentum.
+int dlion_oracle_worker_step(const dlion_oracle_segment* segs, uint32_t nseg,
+                             uint64_t d_pad, uint32_t n_workers, int gdtype,
+                             const void* g, float* m, uint32_t* packed,
+                             float beta1, float beta2, int nthreads) {
+    if (n_workers == 0 || n_workers > 65536) return -1;
+    float* b1 = new float[n_workers];
+    float* b2 = new float[n_workers];
+    for (uint32_t i = 0; i < n_workers; ++i) { b1[i] = beta1; b2[i] = beta2; }
+    const int rc = dlion_oracle_worker_step_ex(segs, nseg, d_pad, n_workers, gdtype, DLION_ORACLE_STATE_F32,
+                                               g, m, packed, b1, b2, nthreads);
+    delete[] b1;
+    delete[] b2;
+    return rc;
 }
 
 // Server side of Algorithm 1 followed by the parameter update of Section 3.2.

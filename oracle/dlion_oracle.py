@@ -24,6 +24,8 @@ MAJORITY = 0
 AVERAGE = 1
 GRAD_F32 = 0
 GRAD_BF16 = 1
+STATE_F32 = 0
+STATE_BF16 = 1
 
 CXXFLAGS = ["-std=c++17", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fopenmp",
             "-fPIC", "-shared"]
@@ -47,6 +49,11 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
         ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32,
         ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
         ctypes.c_float, ctypes.c_float, ctypes.c_int]
+    lib.dlion_oracle_worker_step_ex.restype = ctypes.c_int
+    lib.dlion_oracle_worker_step_ex.argtypes = [
+        ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32,
+        ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
     lib.dlion_oracle_aggregate_apply.restype = ctypes.c_int
     lib.dlion_oracle_aggregate_apply.argtypes = [
         ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32,
@@ -118,6 +125,27 @@ def worker_step(segments, d_pad: int, n_workers: int, g: np.ndarray, m: np.ndarr
         beta1, beta2, nthreads)
     if rc != 0:
         raise ValueError("dlion_oracle_worker_step rejected its arguments")
+
+
+def worker_step_ex(segments, d_pad: int, n_workers: int, g: np.ndarray, m: np.ndarray,
+                   packed: np.ndarray, beta1s, beta2s, nthreads: int = 1,
+                   lib: Optional[ctypes.CDLL] = None) -> None:
+    """General worker side: per-worker betas (Alg. 1, footnote to the inputs) and fp32 or
+    bf16 momentum (``m`` float32, or uint16 holding bf16 bit patterns)."""
+    gdt = {np.dtype(np.float32): GRAD_F32, np.dtype(np.uint16): GRAD_BF16}[g.dtype]
+    mdt = {np.dtype(np.float32): STATE_F32, np.dtype(np.uint16): STATE_BF16}[m.dtype]
+    b1 = np.ascontiguousarray(beta1s, dtype=np.float32)
+    b2 = np.ascontiguousarray(beta2s, dtype=np.float32)
+    _check(g, g.dtype, n_workers * d_pad, "g")
+    _check(m, m.dtype, n_workers * d_pad, "m")
+    _check(packed, np.uint32, n_workers * d_pad // 32, "packed")
+    _check(b1, np.float32, n_workers, "beta1s")
+    _check(b2, np.float32, n_workers, "beta2s")
+    rc = (lib or _get()).dlion_oracle_worker_step_ex(
+        _segs(segments), len(segments), d_pad, n_workers, gdt, mdt, _ptr(g), _ptr(m), _ptr(packed),
+        _ptr(b1), _ptr(b2), nthreads)
+    if rc != 0:
+        raise ValueError("dlion_oracle_worker_step_ex rejected its arguments")
 
 
 def aggregate_apply(segments, d_pad: int, n_workers: int, mode: int, packed: np.ndarray,

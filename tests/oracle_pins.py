@@ -387,8 +387,67 @@ def check_delta_wire_roundtrip(lib):
             assert np.array_equal(xa[~valid], x0[~valid])
 
 
+# ---------------------------------------------------------------- per-worker betas, bf16 momentum
+def check_per_worker_betas(lib):
+    """Algorithm 1 lets each worker set its own beta1, beta2: worker i of a mixed run must be
+    the single-worker run with (beta1_i, beta2_i), bit for bit."""
+    rng = np.random.default_rng(12)
+    segs, d_pad = _flat(700)
+    N, T = 4, 4
+    b1s = [0.9, 0.5, 0.0, 0.95]
+    b2s = [0.99, 0.75, 0.0, 0.95]
+    grads = _rand_grads(rng, T, N, d_pad)
+    m = np.zeros((N, d_pad), np.float32)
+    solo = [np.zeros((1, d_pad), np.float32) for _ in range(N)]
+    for g in grads:
+        packed = np.zeros((N, d_pad // 32), np.uint32)
+        orc.worker_step_ex(segs, d_pad, N, g, m, packed, b1s, b2s, lib=lib)
+        for i in range(N):
+            p1 = np.zeros((1, d_pad // 32), np.uint32)
+            orc.worker_step(segs, d_pad, 1, np.ascontiguousarray(g[i:i + 1]), solo[i], p1, b1s[i], b2s[i],
+                            lib=lib)
+            assert np.array_equal(p1[0], packed[i]) and np.array_equal(solo[i][0], m[i])
+    assert not np.array_equal(m[0], m[1])
+
+
+def check_bf16_momentum_store(lib):
+    """bf16 momentum: arithmetic in binary32, the stored value is the binary32 result rounded to
+    nearest-even bf16 (checked against torch's float32 -> bfloat16 conversion, an independent
+    routine), and the signs are those of the widened state."""
+    import torch
+    rng = np.random.default_rng(13)
+    segs, d_pad = _flat(4096)
+    N = 2
+
+    def to_bits(a32):
+        return torch.from_numpy(a32.copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+
+    def widen(b16):
+        return (b16.astype(np.uint32) << 16).view(np.float32)
+
+    m16 = to_bits(f32(rng.standard_normal((N, d_pad))))
+    g = f32(rng.standard_normal((N, d_pad)))
+    # exact ties: beta2 = 0 makes m' = g; these g sit halfway between two bf16 values
+    g[0, :4] = [1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8), 3.4e38]
+    for b1, b2 in ((0.9, 0.99), (0.5, 0.0)):
+        m32 = widen(m16)
+        p32 = np.zeros((N, d_pad // 32), np.uint32)
+        orc.worker_step(segs, d_pad, N, g, m32, p32, b1, b2, lib=lib)            # fp32-state run from the same start
+        mb = m16.copy()
+        pb = np.zeros((N, d_pad // 32), np.uint32)
+        orc.worker_step_ex(segs, d_pad, N, g, mb, pb, [b1] * N, [b2] * N, lib=lib)
+        assert np.array_equal(pb, p32)                                           # same old m, same signs
+        assert np.array_equal(mb[:, :4096], to_bits(m32)[:, :4096])              # RNE of the fp32 result
+    assert widen(mb)[0, 0] == 1.0 and widen(mb)[0, 1] == 1.0 + 2.0 ** -6 and widen(mb)[0, 2] == -1.0
+    assert np.isinf(widen(mb)[0, 3])                                              # rounds up past the largest bf16
+    nan_state = np.full((1, 128), 0x7FC1, np.uint16)
+    orc.worker_step_ex([(0, 128)], 128, 1, np.zeros((1, 128), np.float32), nan_state,
+                       np.zeros((1, 4), np.uint32), [0.9], [0.99], lib=lib)
+    assert np.isnan(widen(nan_state)).all()
+
+
 ALL_CHECKS = [check_hand_case, check_sign_of_zero_and_tie, check_delta_is_sign_of_blend,
               check_single_worker_is_lion, check_identical_workers, check_beta_zero_is_signsgd,
               check_equal_betas_is_signum, check_counts_bruteforce, check_x_closed_form,
               check_phase_one_contraction, check_padding_untouched, check_wire_bits,
-              check_delta_wire_roundtrip]
+              check_delta_wire_roundtrip, check_per_worker_betas, check_bf16_momentum_store]

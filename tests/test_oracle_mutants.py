@@ -15,8 +15,8 @@ MUTANTS = {
     "delta_negated": ("word |= sign_bit(c) << b;", "word |= sign_bit(-c) << b;"),
     "sign_of_zero_negative": ("return (v >= 0.0f) ? 1u : 0u;", "return (v > 0.0f) ? 1u : 0u;"),
     "bit_order_reversed": ("word |= sign_bit(c) << b;", "word |= sign_bit(c) << (31 - b);"),
-    "momentum_uses_beta1": ("m[idx] = a2 + b2;", "m[idx] = a1 + b1;"),
-    "momentum_drops_gradient": ("m[idx] = a2 + b2;", "m[idx] = a2;"),
+    "momentum_uses_beta1": ("store_state(m, mdtype, idx, a2 + b2);", "store_state(m, mdtype, idx, a1 + b1);"),
+    "momentum_drops_gradient": ("store_state(m, mdtype, idx, a2 + b2);", "store_state(m, mdtype, idx, a2);"),
     "one_minus_beta_dropped": ("const float om2 = 1.0f - beta2;", "const float om2 = 1.0f;"),
     "tie_goes_negative": ("Delta = (S >= 0) ? 1.0f : -1.0f;", "Delta = (S > 0) ? 1.0f : -1.0f;"),
     "sum_is_count": ("const int32_t S = 2 * P - N;", "const int32_t S = P;"),
@@ -39,6 +39,10 @@ MUTANTS = {
     "wire_apply_sign": ("x[j] = xo - u3;", "x[j] = xo + u3;"),
     "wire_tie_negative": ("static_cast<int64_t>(n_workers) >= 0) delta_wire[w] |= 1u << b;",
                           "static_cast<int64_t>(n_workers) > 0) delta_wire[w] |= 1u << b;"),
+    "bf16_store_truncates": ("u += 0x7FFFu + lsb;", "u += 0u;"),
+    "bf16_store_rounds_half_up": ("u += 0x7FFFu + lsb;", "u += 0x8000u;"),
+    "betas_of_worker_zero": ("const float beta1 = beta1s[i], beta2 = beta2s[i];",
+                             "const float beta1 = beta1s[0], beta2 = beta2s[0];"),
     "average_down_bits_floor_log": ("while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;",
                                     "while ((2ull << bits) <= static_cast<uint64_t>(n_workers)) ++bits;"),
 }
