@@ -125,9 +125,9 @@ class ClockSampler:
         return out
 
 
-def bytes_per_param_worker_k1(w) -> float:
+def bytes_per_param_worker_k1(w, state_bytes: int = 4) -> float:
     """Worker-side kernel: gradient + momentum read + momentum write + 1/8 B of signs."""
-    return w.grad_bytes + 4 + 4 + 1 / 8
+    return w.grad_bytes + 2 * state_bytes + 1 / 8
 
 
 def bytes_per_param_k2(w) -> float:
@@ -234,7 +234,10 @@ def run_ours(args):
     ctx = dlion.Dlion(w.segments, D, N, w.beta1, w.beta2, w.lr, w.weight_decay, mode,
                       dlion.GRAD_F32 if w.grad_dtype == "f32" else dlion.GRAD_BF16)
     g = torch.empty(N, D, dtype=gdt, device=dev)
-    m = torch.zeros(N, D, device=dev)
+    sbytes = 2 if args.state == "bf16" else 4
+    if args.state == "bf16":
+        ctx.set_momentum_dtype(dlion.STATE_BF16)
+    m = torch.zeros(N, D, dtype=torch.bfloat16 if args.state == "bf16" else torch.float32, device=dev)
     x = inputs.fill_x0(w, torch.empty(D, device=dev))
     packed = torch.zeros(N, W, dtype=torch.int32, device=dev)
     stream = torch.cuda.current_stream()
@@ -314,13 +317,13 @@ def run_ours(args):
         k1 = statistics.mean(k1_ms)
         k2 = statistics.mean(k2_ms)
         if args.path == "fused":
-            alg_bytes = w.d * (N * (w.grad_bytes + 8) + 8)
+            alg_bytes = w.d * (N * (w.grad_bytes + 2 * sbytes) + 8)
             name = "step_fused_kernel"
         else:
-            alg_bytes = w.d * N * bytes_per_param_worker_k1(w)
+            alg_bytes = w.d * N * bytes_per_param_worker_k1(w, sbytes)
             name = "worker_step_kernel"
         achieved = alg_bytes / (k1 * 1e-3) / 1e9
-        traffic = NCU_TRAFFIC.get((name, kernel_hash()))
+        traffic = NCU_TRAFFIC.get((name, kernel_hash())) if sbytes == 4 and w.grad_dtype == "bf16" else None
         roofline = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_source": peak_src, "frac_of_8tbs_nominal": achieved / 8000.0,
                     "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": k1,
@@ -343,6 +346,7 @@ def run_ours(args):
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "n_workers": N, "d": w.d, "grads": w.grad_dtype,
                        "mode": "average" if mode else "majority", "path": args.path,
+                       "momentum": args.state,
                        "l2": "inputs larger than L2 (no flush needed)" if N * D * (w.grad_bytes + 4) > 4 * 126e6
                              else "working set comparable to L2: latency-bound case",
                        "timed_region": "K steps back to back in one bracket, on the last generated gradients",
@@ -400,6 +404,7 @@ def main():
     ap.add_argument("--n-workers", type=int, default=0, help="override N (the c4 sweep)")
     ap.add_argument("--mode", default=None, choices=["majority", "average"])
     ap.add_argument("--path", default="two_stage", choices=["two_stage", "fused"])
+    ap.add_argument("--state", default="f32", choices=["f32", "bf16"], help="momentum storage")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--e2e-warmup", type=int, default=1)

@@ -25,7 +25,7 @@
  * Memory layout. Every buffer is DEVICE memory owned by the caller, unless a
  * parameter says "host".  Arenas are flat and worker-major:
  *     grads  [N][d_pad]     float or bf16 (dlion_gdtype)
- *     m      [N][d_pad]     float
+ *     m      [N][d_pad]     float (or bf16, see dlion_set_momentum_dtype)
  *     packed [N][d_pad/32]  uint32; bit b of word w is coordinate 32*w+b; 1 = "+1"
  *     x      [d_pad]        float (all workers hold the same x, so one copy)
  * A segment table names the coordinates that are parameters: segment k covers
@@ -68,6 +68,7 @@ typedef enum {
 
 typedef enum { DLION_MAJORITY = 0, DLION_AVERAGE = 1 } dlion_mode;
 typedef enum { DLION_GRAD_F32 = 0, DLION_GRAD_BF16 = 1 } dlion_gdtype;
+typedef enum { DLION_STATE_F32 = 0, DLION_STATE_BF16 = 1 } dlion_sdtype;
 
 typedef struct {
     uint64_t elem_offset; /* first coordinate, in elements, multiple of DLION_ALIGN */
@@ -92,14 +93,29 @@ dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nse
  * Section 5.1): sets eps for the following steps.  lr >= 0 and finite. */
 dlion_status dlion_set_lr(dlion_ctx* ctx, float lr);
 
+/* Storage type of the momentum arenas (default fp32).  With DLION_STATE_BF16 the
+ * m buffers hold bf16: values are widened exactly on load, all arithmetic stays
+ * binary32, and the new momentum is rounded to the nearest bf16, ties to even,
+ * when stored (NaN stays NaN, payload unspecified).  Halves the optimizer state of every worker.
+ * Call before the first step; x stays fp32.  dlion_step_static is fp32 only. */
+dlion_status dlion_set_momentum_dtype(dlion_ctx* ctx, dlion_sdtype sdtype);
+
+/* Algorithm 1 allows every worker its own beta1, beta2 (footnote to its inputs):
+ * sets worker's pair, both in [0,1]; the others keep the values of dlion_init.
+ * beta1 = beta2 makes that worker a Signum worker, beta1 = beta2 = 0 a signSGD
+ * worker (Section 5.1 uses both as D-SIGNUM / D-SignSGD).  Allocates the
+ * per-worker table on first use and copies it synchronously: call it outside
+ * the step loop. */
+dlion_status dlion_set_worker_betas(dlion_ctx* ctx, int worker, float beta1, float beta2);
+
 /* Worker side of Algorithm 1 (the two worker-side assignments; same equations
  * in Section 3.2).  worker = -1: all N workers, pointers are the [N][...]
  * arenas.  worker = i in [0,N): that worker only, pointers are ITS slices
  * (grads[d_pad], m[d_pad], packed[d_pad/32]).
  *   grads   in     gradients g_{i,t}
- *   m       in/out momentum, updated in place
+ *   m       in/out momentum (float, or bf16 after dlion_set_momentum_dtype), updated in place
  *   packed  out    delta_{i,t}, 1 bit per coordinate (Table 1: d bits per worker) */
-dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, float* m,
+dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, void* m,
                                uint32_t* packed, void* cuda_stream);
 
 /* Server side of Algorithm 1 (aggregate(S_t), Section 3.2) fused with the
@@ -145,7 +161,7 @@ uint32_t dlion_delta_planes(const dlion_ctx* ctx);
  * tile of coordinates for all N workers, votes in registers and applies x.
  * Same results as dlion_worker_step(-1) followed by dlion_aggregate_apply.
  *   packed_out  out, nullable: the wire buffer, if the caller still wants it. */
-dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, float* m, float* x,
+dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float* x,
                               uint32_t* packed_out, void* cuda_stream);
 
 /* One whole step with the gradients in HOST memory (pinned memory makes the
@@ -160,7 +176,7 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, float* m, float
  *   host_delta_out  out, host, nullable: copy of delta_wire_dev; needs
  *                   delta_wire_dev.  Complete when cuda_stream's work is.
  * Uses one internal copy stream ordered against cuda_stream by events. */
-dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, float* m, float* x,
+dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, void* m, float* x,
                              uint32_t* packed, void* staging, void* delta_wire_dev,
                              void* host_delta_out, void* cuda_stream);
 

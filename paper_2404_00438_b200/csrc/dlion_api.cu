@@ -116,7 +116,45 @@ dlion_status dlion_set_lr(dlion_ctx* ctx, float lr) {
     return DLION_OK;
 }
 
-dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, float* m,
+dlion_status dlion_set_momentum_dtype(dlion_ctx* ctx, dlion_sdtype sdtype) {
+    if (ctx == nullptr || (sdtype != DLION_STATE_F32 && sdtype != DLION_STATE_BF16)) return DLION_EINVAL;
+    ctx->sdtype = sdtype;
+    return DLION_OK;
+}
+
+dlion_status dlion_set_worker_betas(dlion_ctx* ctx, int worker, float beta1, float beta2) {
+    if (ctx == nullptr || worker < 0 || worker >= static_cast<int>(ctx->n_workers)) return DLION_EINVAL;
+    if (!unit_interval(beta1) || !unit_interval(beta2)) return DLION_EINVAL;
+    const dlion_status ds = device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    if (ctx->betas.empty()) {
+        try {
+            ctx->betas.assign(ctx->n_workers, betas_of(ctx));
+        } catch (...) {
+            return DLION_ENOMEM;
+        }
+        const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->betas_dev),
+                                         sizeof(dlion::Betas) * ctx->n_workers);
+        if (e != cudaSuccess) {
+            ctx->betas.clear();
+            ctx->betas_dev = nullptr;
+            return e == cudaErrorMemoryAllocation ? DLION_ENOMEM : DLION_ECUDA;
+        }
+    }
+    dlion::Betas k;
+    k.b1 = beta1;
+    k.om1 = 1.0f - beta1;
+    k.b2 = beta2;
+    k.om2 = 1.0f - beta2;
+    ctx->betas[worker] = k;
+    if (cudaMemcpy(ctx->betas_dev, ctx->betas.data(), sizeof(dlion::Betas) * ctx->n_workers,
+                   cudaMemcpyHostToDevice) != cudaSuccess) {
+        return DLION_ECUDA;
+    }
+    return DLION_OK;
+}
+
+dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, void* m,
                                uint32_t* packed, void* cuda_stream) {
     if (ctx == nullptr || grads == nullptr || m == nullptr || packed == nullptr) return DLION_EINVAL;
     if (worker < -1 || worker >= static_cast<int>(ctx->n_workers)) return DLION_EINVAL;
@@ -133,6 +171,9 @@ dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, fl
     p.ntiles = ctx->ntiles;
     p.d_pad = ctx->d_pad;
     p.k = betas_of(ctx);
+    p.betas = ctx->betas_dev;
+    p.worker0 = worker < 0 ? 0u : static_cast<uint32_t>(worker);
+    p.m_bf16 = ctx->sdtype == DLION_STATE_BF16 ? 1 : 0;
     const cudaError_t e = dlion::launch_worker_step(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
                                                     static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return DLION_ECUDA;
@@ -167,7 +208,7 @@ dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float
     return DLION_OK;
 }
 
-dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, float* m, float* x,
+dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float* x,
                               uint32_t* packed_out, void* cuda_stream) {
     if (ctx == nullptr || grads == nullptr || m == nullptr || x == nullptr) return DLION_EINVAL;
     if (!aligned(grads, 16) || !aligned(m, 16) || !aligned(x, 16) || !aligned(packed_out, 16)) {
@@ -186,6 +227,8 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, float* m, float
     p.ntiles = ctx->ntiles;
     p.d_pad = ctx->d_pad;
     p.k = betas_of(ctx);
+    p.betas = ctx->betas_dev;
+    p.m_bf16 = ctx->sdtype == DLION_STATE_BF16 ? 1 : 0;
     p.lr = ctx->lr;
     p.wd = ctx->wd;
     p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;

@@ -6,6 +6,7 @@
 // contracted by the compiler, whatever -fmad says.
 #pragma once
 
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -85,6 +86,64 @@ __device__ __forceinline__ float load_grad1(const void* g, unsigned long long id
     }
 }
 
+// Momentum storage: fp32, or bf16 (widened exactly on load; on store the binary32
+// result is rounded to nearest, ties to even, by the hardware conversion; NaN stays
+// NaN).  Two values per conversion: lo goes to the low half of the word.
+__device__ __forceinline__ uint32_t pack_bf16x2_rne(float lo, float hi) {
+    const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+__device__ __forceinline__ uint32_t f32_to_bf16_rne(float f) { return pack_bf16x2_rne(f, 0.0f) & 0xFFFFu; }
+
+template <bool MB16>
+__device__ __forceinline__ float4 load_state4(const void* m, unsigned long long idx) {
+    if constexpr (MB16) {
+        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(m) + idx));
+        return make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
+    } else {
+        return __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(m) + idx));
+    }
+}
+
+template <bool MB16>
+__device__ __forceinline__ void store_state4(void* m, unsigned long long idx, const float4& v) {
+    if constexpr (MB16) {
+        uint2 o;
+        o.x = pack_bf16x2_rne(v.x, v.y);
+        o.y = pack_bf16x2_rne(v.z, v.w);
+        __stcs(reinterpret_cast<uint2*>(static_cast<uint16_t*>(m) + idx), o);
+    } else {
+        __stcs(reinterpret_cast<float4*>(static_cast<float*>(m) + idx), v);
+    }
+}
+
+template <bool MB16>
+__device__ __forceinline__ float load_state1(const void* m, unsigned long long idx) {
+    if constexpr (MB16) {
+        return __uint_as_float(static_cast<uint32_t>(static_cast<const uint16_t*>(m)[idx]) << 16);
+    } else {
+        return static_cast<const float*>(m)[idx];
+    }
+}
+
+template <bool MB16>
+__device__ __forceinline__ void store_state1(void* m, unsigned long long idx, float v) {
+    if constexpr (MB16) static_cast<uint16_t*>(m)[idx] = static_cast<uint16_t>(f32_to_bf16_rne(v));
+    else static_cast<float*>(m)[idx] = v;
+}
+
+// Worker i's coefficients: its row of the per-worker table when one is set
+// (Algorithm 1 lets every worker choose its own beta1, beta2), else the common ones.
+__device__ __forceinline__ Betas betas_of(const Betas* __restrict__ table, const Betas& common,
+                                          unsigned long long worker) {
+    if (table == nullptr) return common;
+    const float4 r = __ldg(reinterpret_cast<const float4*>(table + worker));
+    Betas k;
+    k.b1 = r.x; k.om1 = r.y; k.b2 = r.z; k.om2 = r.w;
+    return k;
+}
+
 // Lane l of each group of 8 lanes holds a nibble (signs of coordinates 4l..4l+3
 // of a 32-coordinate word).  Returns the assembled word in all 8 lanes.
 __device__ __forceinline__ uint32_t gather_word(uint32_t nibble, uint32_t lane) {
@@ -103,7 +162,7 @@ __device__ __forceinline__ uint32_t spread_nibble(uint32_t nibble) {
 // ---- launch parameters ----------------------------------------------------
 struct WorkerParams {
     const void* g;
-    float* m;
+    void* m;                         // float, or bf16 when m_bf16
     uint32_t* packed;
     const SegDev* segs;
     uint32_t nseg;
@@ -111,6 +170,9 @@ struct WorkerParams {
     unsigned long long ntiles;       // tiles per worker
     unsigned long long d_pad;        // elements between consecutive workers in g and m
     Betas k;
+    const Betas* betas;              // per-worker table (device), or null
+    uint32_t worker0;                // id of the first worker this launch covers
+    int m_bf16;
 };
 
 struct AggParams {
@@ -129,7 +191,7 @@ struct AggParams {
 
 struct FusedParams {
     const void* g;
-    float* m;
+    void* m;                         // float, or bf16 when m_bf16
     float* x;
     uint32_t* packed;                // nullable
     const SegDev* segs;
@@ -138,6 +200,8 @@ struct FusedParams {
     unsigned long long ntiles;
     unsigned long long d_pad;
     Betas k;
+    const Betas* betas;              // per-worker table (device), or null
+    int m_bf16;
     float lr, wd;
     int average;
 };

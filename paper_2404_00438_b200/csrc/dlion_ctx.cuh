@@ -16,6 +16,9 @@ struct dlion_ctx {
     float beta1 = 0, beta2 = 0, lr = 0, wd = 0;
     dlion_mode mode = DLION_MAJORITY;
     dlion_gdtype gdtype = DLION_GRAD_F32;
+    dlion_sdtype sdtype = DLION_STATE_F32;
+    std::vector<dlion::Betas> betas;         // per-worker rows (empty until one is set)
+    dlion::Betas* betas_dev = nullptr;
     int device = -1;
     int sm_count = 0;
     uint64_t launches = 0;

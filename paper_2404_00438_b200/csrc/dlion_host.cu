@@ -21,7 +21,7 @@ cudaError_t ensure_pipeline(dlion_ctx* c) {
 
 extern "C" {
 
-dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, float* m, float* x,
+dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, void* m, float* x,
                              uint32_t* packed, void* staging, void* delta_wire_dev,
                              void* host_delta_out, void* cuda_stream) {
     if (ctx == nullptr || host_grads == nullptr || m == nullptr || x == nullptr || packed == nullptr ||
@@ -40,6 +40,7 @@ dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, float* m, f
 
     cudaStream_t main = static_cast<cudaStream_t>(cuda_stream);
     const size_t gsz = ctx->gdtype == DLION_GRAD_BF16 ? 2 : 4;
+    const size_t msz = ctx->sdtype == DLION_STATE_BF16 ? 2 : 4;
     const size_t slice = static_cast<size_t>(ctx->d_pad) * gsz;        // one worker's gradients
     const size_t words = static_cast<size_t>(ctx->d_pad / 32);
     const char* hsrc = static_cast<const char*>(host_grads);
@@ -58,7 +59,7 @@ dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, float* m, f
         if (cudaEventRecord(ctx->copied[b], ctx->copy_stream) != cudaSuccess) return DLION_ECUDA;
         if (cudaStreamWaitEvent(main, ctx->copied[b], 0) != cudaSuccess) return DLION_ECUDA;
         const dlion_status st = dlion_worker_step(ctx, static_cast<int>(i), stage + b * slice,
-                                                  m + static_cast<size_t>(i) * ctx->d_pad,
+                                                  static_cast<char*>(m) + static_cast<size_t>(i) * ctx->d_pad * msz,
                                                   packed + static_cast<size_t>(i) * words, main);
         if (st != DLION_OK) return st;
         if (cudaEventRecord(ctx->consumed[b], main) != cudaSuccess) return DLION_ECUDA;
@@ -162,6 +163,7 @@ const char* dlion_status_str(dlion_status s) {
 void dlion_destroy(dlion_ctx* ctx) {
     if (ctx == nullptr) return;
     if (ctx->segs_dev != nullptr) cudaFree(ctx->segs_dev);
+    if (ctx->betas_dev != nullptr) cudaFree(ctx->betas_dev);
     for (int k = 0; k < 2; ++k) {
         if (ctx->copied[k] != nullptr) cudaEventDestroy(ctx->copied[k]);
         if (ctx->consumed[k] != nullptr) cudaEventDestroy(ctx->consumed[k]);

@@ -30,7 +30,7 @@ struct RawGrad4 { float4 v; };            // four gradients as stored
 template <>
 struct RawGrad4<true> { uint2 v; };
 
-template <bool BF16>
+template <bool BF16, bool MB16>
 struct WorkerRegs {                       // one worker's gradients and momenta of my coordinates
     RawGrad4<BF16> g[kChunksPerWarp];
     float4 m[kChunksPerWarp];
@@ -42,7 +42,7 @@ struct WorkerRegs {                       // one worker's gradients and momenta 
             } else {
                 g[u].v = __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(p.g) + at + u * kChunk));
             }
-            m[u] = __ldcs(reinterpret_cast<const float4*>(p.m + at + u * kChunk));
+            m[u] = load_state4<MB16>(p.m, at + u * kChunk);
         }
     }
     __device__ __forceinline__ float4 grad(int u) const {
@@ -56,18 +56,20 @@ struct WorkerRegs {                       // one worker's gradients and momenta 
 
 // Worker-side update of my coordinates for one worker: momenta stored, votes
 // added to cnt (one byte per coordinate), wire words written if requested.
-template <bool BF16>
-__device__ __forceinline__ void consume(const FusedParams& p, WorkerRegs<BF16>& r, unsigned long long at,
-                                        uint32_t* wire_words, uint32_t lane, uint32_t (&cnt)[kChunksPerWarp]) {
+template <bool BF16, bool MB16>
+__device__ __forceinline__ void consume(const FusedParams& p, WorkerRegs<BF16, MB16>& r, uint32_t worker,
+                                        unsigned long long at, uint32_t* wire_words, uint32_t lane,
+                                        uint32_t (&cnt)[kChunksPerWarp]) {
+    const Betas k = betas_of(p.betas, p.k, worker);
     uint32_t mine = 0;
 #pragma unroll
     for (int u = 0; u < kChunksPerWarp; ++u) {
         const float4 g = r.grad(u);
-        uint32_t nib = lion_coord(g.x, r.m[u].x, p.k);
-        nib |= lion_coord(g.y, r.m[u].y, p.k) << 1;
-        nib |= lion_coord(g.z, r.m[u].z, p.k) << 2;
-        nib |= lion_coord(g.w, r.m[u].w, p.k) << 3;
-        __stcs(reinterpret_cast<float4*>(p.m + at + u * kChunk), r.m[u]);
+        uint32_t nib = lion_coord(g.x, r.m[u].x, k);
+        nib |= lion_coord(g.y, r.m[u].y, k) << 1;
+        nib |= lion_coord(g.z, r.m[u].z, k) << 2;
+        nib |= lion_coord(g.w, r.m[u].w, k) << 3;
+        store_state4<MB16>(p.m, at + u * kChunk, r.m[u]);
         cnt[u] += spread_nibble(nib);
         if (wire_words != nullptr) {                              // block-uniform
             const uint32_t w = gather_word(nib, lane);
@@ -80,7 +82,7 @@ __device__ __forceinline__ void consume(const FusedParams& p, WorkerRegs<BF16>& 
 }
 
 // Last tile of a segment: every access guarded, one chunk at a time.
-template <bool BF16, bool AVG>
+template <bool BF16, bool AVG, bool MB16>
 __device__ __noinline__ void ragged_tile(const FusedParams& p, const TileRef t, uint32_t in_tile,
                                          unsigned long long e0, uint32_t lane, uint32_t thr,
                                          const float* avg_table) {
@@ -95,12 +97,13 @@ __device__ __noinline__ void ragged_tile(const FusedParams& p, const TileRef t, 
         uint32_t c4 = 0;
         for (uint32_t i = 0; i < n; ++i) {
             const unsigned long long e = i * p.d_pad + e0 + u * kChunk;
+            const Betas k = betas_of(p.betas, p.k, i);
             uint32_t nib = 0;
             for (uint32_t q = 0; q < mine_n; ++q) {
                 const float g = load_grad1<BF16>(p.g, e + q);
-                float m = p.m[e + q];
-                nib |= lion_coord(g, m, p.k) << q;
-                p.m[e + q] = m;
+                float m = load_state1<MB16>(p.m, e + q);
+                nib |= lion_coord(g, m, k) << q;
+                store_state1<MB16>(p.m, e + q, m);
             }
             c4 += spread_nibble(nib);
             if (p.packed != nullptr) {
@@ -117,7 +120,7 @@ __device__ __noinline__ void ragged_tile(const FusedParams& p, const TileRef t, 
     }
 }
 
-template <bool BF16, bool AVG>
+template <bool BF16, bool AVG, bool MB16>
 __global__ void __launch_bounds__(kThreads, 2)
 step_fused_kernel(const __grid_constant__ FusedParams p) {
     __shared__ float avg_table[256];
@@ -151,17 +154,17 @@ step_fused_kernel(const __grid_constant__ FusedParams p) {
                 xv[u] = __ldcs(reinterpret_cast<const float4*>(p.x + e0 + u * kChunk));
             }
             uint32_t* wire = p.packed == nullptr ? nullptr : p.packed + (t.base + in_tile) / 32;
-            WorkerRegs<BF16> a, b;
+            WorkerRegs<BF16, MB16> a, b;
             a.load(p, e0);
             uint32_t i = 0;
             for (; i + 2 <= n; i += 2) {
                 b.load(p, (i + 1) * p.d_pad + e0);
-                consume<BF16>(p, a, i * p.d_pad + e0, wire == nullptr ? nullptr : wire + i * w_stride, lane, cnt);
+                consume<BF16, MB16>(p, a, i, i * p.d_pad + e0, wire == nullptr ? nullptr : wire + i * w_stride, lane, cnt);
                 if (i + 2 < n) a.load(p, (i + 2) * p.d_pad + e0);
-                consume<BF16>(p, b, (i + 1) * p.d_pad + e0, wire == nullptr ? nullptr : wire + (i + 1) * w_stride,
+                consume<BF16, MB16>(p, b, i + 1, (i + 1) * p.d_pad + e0, wire == nullptr ? nullptr : wire + (i + 1) * w_stride,
                               lane, cnt);
             }
-            if (i < n) consume<BF16>(p, a, i * p.d_pad + e0, wire == nullptr ? nullptr : wire + i * w_stride, lane, cnt);
+            if (i < n) consume<BF16, MB16>(p, a, i, i * p.d_pad + e0, wire == nullptr ? nullptr : wire + i * w_stride, lane, cnt);
 #pragma unroll
             for (int u = 0; u < kChunksPerWarp; ++u) {
                 float4 v = xv[u];
@@ -172,18 +175,18 @@ step_fused_kernel(const __grid_constant__ FusedParams p) {
                 __stcs(reinterpret_cast<float4*>(p.x + e0 + u * kChunk), v);
             }
         } else {
-            ragged_tile<BF16, AVG>(p, t, in_tile, e0, lane, thr, avg_table);
+            ragged_tile<BF16, AVG, MB16>(p, t, in_tile, e0, lane, thr, avg_table);
         }
     }
 }
 
-template <bool BF16>
+template <bool BF16, bool MB16>
 cudaError_t launch(const FusedParams& p, cudaStream_t s) {
     if (p.ntiles == 0) return cudaSuccess;
     if (p.average) {
-        step_fused_kernel<BF16, true><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
+        step_fused_kernel<BF16, true, MB16><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
     } else {
-        step_fused_kernel<BF16, false><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
+        step_fused_kernel<BF16, false, MB16><<<grid_for(p.ntiles), kThreads, 0, s>>>(p);
     }
     return cudaGetLastError();
 }
@@ -192,7 +195,8 @@ cudaError_t launch(const FusedParams& p, cudaStream_t s) {
 
 cudaError_t launch_step_fused(const FusedParams& p, bool bf16, int sm_count, cudaStream_t s) {
     (void)sm_count;
-    return bf16 ? launch<true>(p, s) : launch<false>(p, s);
+    if (p.m_bf16) return bf16 ? launch<true, true>(p, s) : launch<false, true>(p, s);
+    return bf16 ? launch<true, false>(p, s) : launch<false, false>(p, s);
 }
 
 }  // namespace dlion

@@ -111,6 +111,9 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
     wp.k.om1 = 1.0f - beta1;
     wp.k.b2 = beta2;
     wp.k.om2 = 1.0f - beta2;
+    wp.betas = nullptr;
+    wp.worker0 = 0;
+    wp.m_bf16 = 0;
     if (dlion::launch_worker_step(wp, gdtype == DLION_GRAD_BF16, pd.sm_count, s) != cudaSuccess) {
         return DLION_ECUDA;
     }

@@ -27,7 +27,7 @@ constexpr int kThreads = 256;            // 8 warps x 512 coordinates = one tile
 constexpr int kChunksPerWarp = 4;
 
 // (Parameters are taken by value on purpose: marking them __grid_constant__ measured 6 % slower here.)
-template <bool BF16>
+template <bool BF16, bool MB16>
 __global__ void __launch_bounds__(kThreads)
 worker_step_kernel(const WorkerParams p) {
     const uint32_t lane = threadIdx.x & 31u;
@@ -39,6 +39,7 @@ worker_step_kernel(const WorkerParams p) {
         const unsigned long long worker = item / p.ntiles;
         const TileRef t = find_tile(p.segs, p.nseg, item - worker * p.ntiles);
         const unsigned long long wbase = worker * p.d_pad;         // element offset of this worker
+        const Betas k = betas_of(p.betas, p.k, p.worker0 + worker);
         const uint32_t in_tile = warp * (kChunksPerWarp * kChunk); // first coordinate of this warp
         uint32_t* words = p.packed + worker * w_stride + (t.base + in_tile) / 32;
 
@@ -49,16 +50,16 @@ worker_step_kernel(const WorkerParams p) {
 #pragma unroll
             for (int u = 0; u < kChunksPerWarp; ++u) {
                 g[u] = load_grad4<BF16>(p.g, e0 + u * kChunk);
-                m[u] = __ldcs(reinterpret_cast<const float4*>(p.m + e0 + u * kChunk));
+                m[u] = load_state4<MB16>(p.m, e0 + u * kChunk);
             }
             uint32_t mine = 0;
 #pragma unroll
             for (int u = 0; u < kChunksPerWarp; ++u) {
-                uint32_t nib = lion_coord(g[u].x, m[u].x, p.k);
-                nib |= lion_coord(g[u].y, m[u].y, p.k) << 1;
-                nib |= lion_coord(g[u].z, m[u].z, p.k) << 2;
-                nib |= lion_coord(g[u].w, m[u].w, p.k) << 3;
-                __stcs(reinterpret_cast<float4*>(p.m + e0 + u * kChunk), m[u]);
+                uint32_t nib = lion_coord(g[u].x, m[u].x, k);
+                nib |= lion_coord(g[u].y, m[u].y, k) << 1;
+                nib |= lion_coord(g[u].z, m[u].z, k) << 2;
+                nib |= lion_coord(g[u].w, m[u].w, k) << 3;
+                store_state4<MB16>(p.m, e0 + u * kChunk, m[u]);
                 const uint32_t w = gather_word(nib, lane);
                 if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
             }
@@ -75,18 +76,18 @@ worker_step_kernel(const WorkerParams p) {
                 uint32_t nib = 0;
                 if (j0 + 4 <= t.valid) {
                     float4 g = load_grad4<BF16>(p.g, e);
-                    float4 m = __ldcs(reinterpret_cast<const float4*>(p.m + e));
-                    nib = lion_coord(g.x, m.x, p.k);
-                    nib |= lion_coord(g.y, m.y, p.k) << 1;
-                    nib |= lion_coord(g.z, m.z, p.k) << 2;
-                    nib |= lion_coord(g.w, m.w, p.k) << 3;
-                    __stcs(reinterpret_cast<float4*>(p.m + e), m);
+                    float4 m = load_state4<MB16>(p.m, e);
+                    nib = lion_coord(g.x, m.x, k);
+                    nib |= lion_coord(g.y, m.y, k) << 1;
+                    nib |= lion_coord(g.z, m.z, k) << 2;
+                    nib |= lion_coord(g.w, m.w, k) << 3;
+                    store_state4<MB16>(p.m, e, m);
                 } else {
                     for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
                         const float g = load_grad1<BF16>(p.g, e + q);
-                        float m = p.m[e + q];
-                        nib |= lion_coord(g, m, p.k) << q;
-                        p.m[e + q] = m;
+                        float m = load_state1<MB16>(p.m, e + q);
+                        nib |= lion_coord(g, m, k) << q;
+                        store_state1<MB16>(p.m, e + q, m);
                     }
                 }
                 const uint32_t w = gather_word(nib, lane);
@@ -99,11 +100,11 @@ worker_step_kernel(const WorkerParams p) {
     }
 }
 
-template <bool BF16>
+template <bool BF16, bool MB16>
 cudaError_t launch(const WorkerParams& p, cudaStream_t s) {
     const unsigned long long n_items = p.ntiles * p.n_workers;
     if (n_items == 0) return cudaSuccess;
-    worker_step_kernel<BF16><<<grid_for(n_items), kThreads, 0, s>>>(p);
+    worker_step_kernel<BF16, MB16><<<grid_for(n_items), kThreads, 0, s>>>(p);
     return cudaGetLastError();
 }
 
@@ -111,7 +112,8 @@ cudaError_t launch(const WorkerParams& p, cudaStream_t s) {
 
 cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s) {
     (void)sm_count;
-    return bf16 ? launch<true>(p, s) : launch<false>(p, s);
+    if (p.m_bf16) return bf16 ? launch<true, true>(p, s) : launch<false, true>(p, s);
+    return bf16 ? launch<true, false>(p, s) : launch<false, false>(p, s);
 }
 
 }  // namespace dlion

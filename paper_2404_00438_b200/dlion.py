@@ -17,11 +17,13 @@ from . import build as _build
 
 MAJORITY, AVERAGE = 0, 1
 GRAD_F32, GRAD_BF16 = 0, 1
+STATE_F32, STATE_BF16 = 0, 1
 ALIGN = 128
 MAX_WORKERS = 255
 OK, EINVAL, EALIGN, ENOMEM, ECUDA, ESTATE = range(6)
 
-EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_worker_step",
+EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_set_momentum_dtype",
+           "dlion_set_worker_betas", "dlion_worker_step",
            "dlion_aggregate_apply", "dlion_aggregate", "dlion_apply_delta", "dlion_delta_planes",
            "dlion_step_fused", "dlion_step_host", "dlion_step_static",
            "dlion_wire_bytes",
@@ -53,6 +55,10 @@ def _load() -> ctypes.CDLL:
     lib.dlion_init.restype = i32
     lib.dlion_set_lr.argtypes = [vp, f32]
     lib.dlion_set_lr.restype = i32
+    lib.dlion_set_momentum_dtype.argtypes = [vp, i32]
+    lib.dlion_set_momentum_dtype.restype = i32
+    lib.dlion_set_worker_betas.argtypes = [vp, i32, f32, f32]
+    lib.dlion_set_worker_betas.restype = i32
     lib.dlion_worker_step.argtypes = [vp, i32, vp, vp, vp, vp]
     lib.dlion_worker_step.restype = i32
     lib.dlion_aggregate_apply.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -148,6 +154,13 @@ class Dlion:
 
     def set_lr(self, lr: float) -> None:
         self._check(_lib.dlion_set_lr(self._ctx, lr), "dlion_set_lr")
+
+    def set_momentum_dtype(self, sdtype: int) -> None:
+        self._check(_lib.dlion_set_momentum_dtype(self._ctx, int(sdtype)), "dlion_set_momentum_dtype")
+
+    def set_worker_betas(self, worker: int, beta1: float, beta2: float) -> None:
+        self._check(_lib.dlion_set_worker_betas(self._ctx, int(worker), beta1, beta2),
+                    "dlion_set_worker_betas")
 
     def worker_step(self, worker: int, grads: torch.Tensor, m: torch.Tensor,
                     packed: torch.Tensor) -> None:

@@ -210,3 +210,80 @@ def test_aggregate_then_apply_delta(dl, n, mode):
     gp.compare("x after apply_delta", x.cpu().numpy(), x_ref, True)
     assert torch.equal(x, x_one)
     ctx.destroy()
+
+
+# ---------------------------------------------------------------- per-worker betas, bf16 momentum
+def _bf16_ulp_diff(a: np.ndarray, b: np.ndarray) -> int:
+    """Distance in bf16 units in the last place between two arrays of bf16 bit patterns."""
+    def key(u):
+        i = u.astype(np.int64)
+        return np.where(i & 0x8000, -(i & 0x7FFF), i)
+    return int(np.abs(key(a) - key(b)).max()) if a.size else 0
+
+
+@pytest.mark.parametrize("state", ["f32", "bf16"])
+@pytest.mark.parametrize("path", ["two_stage", "per_worker", "fused"])
+@pytest.mark.parametrize("gd", ["f32", "bf16"])
+def test_per_worker_betas_and_momentum_dtype(dl, state, path, gd):
+    """Each worker with its own (beta1, beta2) -- including a Signum and a signSGD worker --
+    and the momentum kept in fp32 or bf16.  Tolerance: signs, counts and Delta exact; fp32
+    state 2 ulp; bf16 state 1 bf16 ulp (observed: identical bits)."""
+    from oracle import dlion_oracle as orc
+    n = 5
+    b1s = [0.9, 0.5, 0.95, 0.0, 0.8]
+    b2s = [0.99, 0.75, 0.95, 0.0, 0.999]
+    w = inputs.custom(RAGGED + [2 * 4096 + 77], n, AVG, gd, scale=1.0 if gd == "f32" else 1e-3,
+                      lr=1e-3, weight_decay=0.5, zero_frac=0.02)
+    dev = torch.device("cuda:0")
+    D, W = w.d_pad, w.d_pad // 32
+    ctx = gp.make_ctx(dl, w)
+    for i in range(n):
+        ctx.set_worker_betas(i, b1s[i], b2s[i])
+    if state == "bf16":
+        ctx.set_momentum_dtype(dl.STATE_BF16)
+    mt = torch.bfloat16 if state == "bf16" else torch.float32
+    x0 = inputs.fill_x0(w, torch.empty(D))
+    m_ref = np.zeros((n, D), np.uint16 if state == "bf16" else np.float32)
+    x_ref = x0.numpy().copy()
+    m = torch.zeros(n, D, dtype=mt, device=dev)
+    x = x0.to(dev)
+    packed = torch.zeros(n, W, dtype=torch.int32, device=dev)
+    for t in range(4):
+        g_cpu = inputs.fill_grads(w, t, torch.empty(n, D, dtype=inputs.grad_torch_dtype(w)))
+        p_ref = np.zeros((n, W), np.uint32)
+        orc.worker_step_ex(w.segments, D, n, inputs.as_numpy_grads(g_cpu), m_ref, p_ref, b1s, b2s)
+        orc.aggregate_apply(w.segments, D, n, AVG, p_ref, x_ref, w.lr, w.weight_decay)
+        g = g_cpu.to(dev)
+        packed.zero_()
+        if path == "fused":
+            ctx.step_fused(g, m, x, packed)
+        else:
+            if path == "per_worker":
+                for i in range(n):
+                    ctx.worker_step(i, g[i], m[i], packed[i])
+            else:
+                ctx.worker_step(-1, g, m, packed)
+            ctx.aggregate_apply(packed, x)
+        torch.cuda.synchronize()
+        gp.compare(f"step {t} packed", packed.cpu().numpy().view(np.uint32), p_ref, True)
+        if state == "bf16":
+            got = m.cpu().view(torch.int16).numpy().view(np.uint16)
+            assert _bf16_ulp_diff(got, m_ref) <= 1
+            assert np.array_equal(got, m_ref)
+        else:
+            assert gp.compare(f"step {t} m", m.cpu().numpy(), m_ref, False) == 0
+        assert gp.compare(f"step {t} x", x.cpu().numpy(), x_ref, False) == 0
+    ctx.destroy()
+
+
+def test_new_setters_reject_bad_arguments(dl):
+    w = inputs.custom([5000], 2, MAJ, "f32")
+    ctx = gp.make_ctx(dl, w)
+    for args in ((-1, 0.9, 0.99), (2, 0.9, 0.99), (0, 1.5, 0.99), (0, 0.9, float("nan"))):
+        with pytest.raises(dl.DlionError) as e:
+            ctx.set_worker_betas(*args)
+        assert e.value.status == dl.EINVAL
+    with pytest.raises(dl.DlionError) as e:
+        ctx.set_momentum_dtype(7)
+    assert e.value.status == dl.EINVAL
+    ctx.destroy()
