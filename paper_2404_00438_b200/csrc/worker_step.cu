@@ -32,12 +32,11 @@ __global__ void __launch_bounds__(kThreads)
 worker_step_kernel(const WorkerParams p) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
-    const unsigned long long n_items = p.ntiles * p.n_workers;
     const unsigned long long w_stride = p.d_pad / 32;
+    const unsigned long long worker = blockIdx.y;                  // grid: x = tile (fastest), y = worker
 
-    for (unsigned long long item = blockIdx.x; item < n_items; item += gridDim.x) {
-        const unsigned long long worker = item / p.ntiles;
-        const TileRef t = find_tile(p.segs, p.nseg, item - worker * p.ntiles);
+    for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
+        const TileRef t = find_tile(p.segs, p.nseg, tile);
         const unsigned long long wbase = worker * p.d_pad;         // element offset of this worker
         const Betas k = betas_of(p.betas, p.k, p.worker0 + worker);
         const uint32_t in_tile = warp * (kChunksPerWarp * kChunk); // first coordinate of this warp
@@ -102,9 +101,9 @@ worker_step_kernel(const WorkerParams p) {
 
 template <bool BF16, bool MB16>
 cudaError_t launch(const WorkerParams& p, cudaStream_t s) {
-    const unsigned long long n_items = p.ntiles * p.n_workers;
-    if (n_items == 0) return cudaSuccess;
-    worker_step_kernel<BF16, MB16><<<grid_for(n_items), kThreads, 0, s>>>(p);
+    if (p.ntiles == 0 || p.n_workers == 0) return cudaSuccess;
+    const dim3 grid(grid_for(p.ntiles), p.n_workers);               // blocks are dispatched x first: worker-major item order
+    worker_step_kernel<BF16, MB16><<<grid, kThreads, 0, s>>>(p);
     return cudaGetLastError();
 }
 
