@@ -82,8 +82,8 @@ dlion_status dlion_check_layout(const dlion_segment* segs, uint32_t nseg, uint64
 
 /* Algorithm 1 "Inputs": N, beta1, beta2 in [0,1], learning rate eps >= 0, weight
  * decay lambda >= 0, and the aggregation rule (Section 3.2).  Validates, then
- * copies the segment table to the current device (a few bytes per segment; the
- * only device memory the library owns).  *out is set only on DLION_OK.
+ * copies the segment table and a 16-byte row per 4096-coordinate tile to the
+ * current device (the only device memory the library owns: 0.1 % of x's size).  *out is set only on DLION_OK.
  * nseg = 1 with elem_offset = 0 describes a flat vector of d = numel. */
 dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nseg,
                         uint64_t d_pad, uint32_t n_workers, float beta1, float beta2,

@@ -76,7 +76,7 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
     };
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
         if (t.valid != kTile) {
             if (!have_table) fill_table();
             ragged_tile<PLANES, AVG, COUNTS>(p, t, warp, lane, thr, avg_table);

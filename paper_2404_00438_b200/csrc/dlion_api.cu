@@ -106,6 +106,35 @@ dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nse
         delete c;
         return DLION_ECUDA;
     }
+    if (tiles != 0) {
+        std::vector<dlion::TileRow> trows;
+        try {
+            trows.reserve(tiles);
+        } catch (...) {
+            cudaFree(c->segs_dev);
+            delete c;
+            return DLION_ENOMEM;
+        }
+        for (uint32_t s = 0; s < nseg; ++s) {
+            for (uint64_t off = 0; off < segs[s].numel; off += dlion::kTile) {
+                dlion::TileRow r;
+                r.base = segs[s].elem_offset + off;
+                r.valid = static_cast<uint32_t>(segs[s].numel - off < dlion::kTile ? segs[s].numel - off : dlion::kTile);
+                r.reserved = 0;
+                trows.push_back(r);
+            }
+        }
+        e = cudaMalloc(reinterpret_cast<void**>(&c->tiles_dev), sizeof(dlion::TileRow) * tiles);
+        if (e == cudaSuccess) {
+            e = cudaMemcpy(c->tiles_dev, trows.data(), sizeof(dlion::TileRow) * tiles, cudaMemcpyHostToDevice);
+        }
+        if (e != cudaSuccess) {
+            if (c->tiles_dev != nullptr) cudaFree(c->tiles_dev);
+            cudaFree(c->segs_dev);
+            delete c;
+            return e == cudaErrorMemoryAllocation ? DLION_ENOMEM : DLION_ECUDA;
+        }
+    }
     *out = c;
     return DLION_OK;
 }
@@ -166,6 +195,7 @@ dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, vo
     p.m = m;
     p.packed = packed;
     p.segs = ctx->segs_dev;
+    p.tiles = ctx->tiles_dev;
     p.nseg = ctx->nseg;
     p.n_workers = worker < 0 ? ctx->n_workers : 1u;
     p.ntiles = ctx->ntiles;
@@ -195,6 +225,7 @@ dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float
     p.delta_bits = delta_bits_out;
     p.count = count_out;
     p.segs = ctx->segs_dev;
+    p.tiles = ctx->tiles_dev;
     p.nseg = ctx->nseg;
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
@@ -222,6 +253,7 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float*
     p.x = x;
     p.packed = packed_out;
     p.segs = ctx->segs_dev;
+    p.tiles = ctx->tiles_dev;
     p.nseg = ctx->nseg;
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;

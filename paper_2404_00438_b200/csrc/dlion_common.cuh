@@ -31,10 +31,25 @@ struct TileRef {
     uint32_t valid;            // parameters in the tile, 1..kTile
 };
 
+// Optional one-row-per-tile table (built by dlion_init): turns the lookup into a
+// single 16-byte load.  Contexts without it (the fixed-scratch step) search.
+struct TileRow {
+    unsigned long long base;   // arena index of the tile's first coordinate
+    uint32_t valid;            // parameters in the tile, 1..kTile
+    uint32_t reserved;
+};
+
 // Largest s with segs[s].first_tile <= tile (segments with numel = 0 own no tile
 // and are never selected because the next row has the same first_tile).
-__device__ __forceinline__ TileRef find_tile(const SegDev* __restrict__ segs, uint32_t nseg,
-                                             unsigned long long tile) {
+__device__ __forceinline__ TileRef find_tile(const TileRow* __restrict__ tiles, const SegDev* __restrict__ segs,
+                                             uint32_t nseg, unsigned long long tile) {
+    if (tiles != nullptr) {
+        const uint4 r = __ldg(reinterpret_cast<const uint4*>(tiles + tile));
+        TileRef t;
+        t.base = static_cast<unsigned long long>(r.x) | (static_cast<unsigned long long>(r.y) << 32);
+        t.valid = r.z;
+        return t;
+    }
     uint32_t lo = 0, hi = nseg;          // answer in [lo, hi)
     while (hi - lo > 1) {
         const uint32_t mid = (lo + hi) >> 1;
@@ -165,6 +180,7 @@ struct WorkerParams {
     void* m;                         // float, or bf16 when m_bf16
     uint32_t* packed;
     const SegDev* segs;
+    const TileRow* tiles;            // per-tile rows (device), or null: search segs
     uint32_t nseg;
     uint32_t n_workers;              // workers this launch covers (1 for a single-worker call)
     unsigned long long ntiles;       // tiles per worker
@@ -181,6 +197,7 @@ struct AggParams {
     uint32_t* delta_bits;            // nullable
     uint8_t* count;                  // nullable
     const SegDev* segs;
+    const TileRow* tiles;            // per-tile rows (device), or null: search segs
     uint32_t nseg;
     uint32_t n_workers;
     unsigned long long ntiles;
@@ -195,6 +212,7 @@ struct FusedParams {
     float* x;
     uint32_t* packed;                // nullable
     const SegDev* segs;
+    const TileRow* tiles;            // per-tile rows (device), or null: search segs
     uint32_t nseg;
     uint32_t n_workers;
     unsigned long long ntiles;
@@ -212,6 +230,7 @@ struct WireParams {                  // server-only aggregate / worker-side appl
     const uint32_t* wire_in;         // apply: the broadcast message
     float* x;                        // apply: parameters
     const SegDev* segs;
+    const TileRow* tiles;            // per-tile rows (device), or null: search segs
     uint32_t nseg;
     uint32_t n_workers;
     unsigned long long ntiles;

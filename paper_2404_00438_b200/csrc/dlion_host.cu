@@ -93,6 +93,7 @@ dlion_status dlion_aggregate(dlion_ctx* ctx, const uint32_t* packed, uint32_t* d
     p.packed = packed;
     p.wire_out = delta_wire;
     p.segs = ctx->segs_dev;
+    p.tiles = ctx->tiles_dev;
     p.nseg = ctx->nseg;
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
@@ -113,6 +114,7 @@ dlion_status dlion_apply_delta(dlion_ctx* ctx, const uint32_t* delta_wire, float
     p.wire_in = delta_wire;
     p.x = x;
     p.segs = ctx->segs_dev;
+    p.tiles = ctx->tiles_dev;
     p.nseg = ctx->nseg;
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
@@ -163,6 +165,7 @@ const char* dlion_status_str(dlion_status s) {
 void dlion_destroy(dlion_ctx* ctx) {
     if (ctx == nullptr) return;
     if (ctx->segs_dev != nullptr) cudaFree(ctx->segs_dev);
+    if (ctx->tiles_dev != nullptr) cudaFree(ctx->tiles_dev);
     if (ctx->betas_dev != nullptr) cudaFree(ctx->betas_dev);
     for (int k = 0; k < 2; ++k) {
         if (ctx->copied[k] != nullptr) cudaEventDestroy(ctx->copied[k]);

@@ -138,7 +138,7 @@ step_fused_kernel(const __grid_constant__ FusedParams p) {
     const unsigned long long w_stride = p.d_pad / 32;
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
         const uint32_t in_tile = warp * (kChunksPerWarp * kChunk);
         if (in_tile >= t.valid) continue;                          // warp-uniform
         const unsigned long long e0 = t.base + in_tile + lane * 4;  // my first coordinate (chunk 0)

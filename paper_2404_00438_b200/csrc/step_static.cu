@@ -103,6 +103,7 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
     wp.m = m;
     wp.packed = wire;
     wp.segs = row;
+    wp.tiles = nullptr;
     wp.nseg = 1;
     wp.n_workers = n_workers;
     wp.ntiles = ntiles;
@@ -124,6 +125,7 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
     ap.delta_bits = nullptr;
     ap.count = nullptr;
     ap.segs = row;
+    ap.tiles = nullptr;
     ap.nseg = 1;
     ap.n_workers = n_workers;
     ap.ntiles = ntiles;

@@ -29,7 +29,7 @@ aggregate_kernel(const __grid_constant__ WireParams p) {
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t thr = (p.n_workers + 1u) >> 1;
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
         const uint32_t my0 = warp * kWarpSpan + lane * 32;          // first coordinate of my word
         if (my0 >= t.valid) continue;                               // my word holds no parameter
         const uint32_t nbits = t.valid - my0 >= 32u ? 32u : t.valid - my0;
@@ -57,7 +57,7 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
     bool have_table = !AVG;
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
         const uint32_t w0 = warp * kWarpSpan;
         if (w0 >= t.valid) continue;                                // warp-uniform
         const bool full = w0 + kWarpSpan <= t.valid;
