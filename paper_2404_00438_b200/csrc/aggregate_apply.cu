@@ -24,7 +24,7 @@ namespace dlion {
 namespace {
 
 constexpr int kThreads = 128;             // 4 warps x 1024 coordinates = one tile
-constexpr int kMinBlocks = 6;             // register budget: 6 blocks (24 warps) per SM
+constexpr int kMinBlocks = 6;             // register budget: 6 blocks (24 warps) per SM; 4 once N >= 64
 // Last tile of a segment: every access guarded against the segment's end.
 template <int PLANES, bool AVG, bool COUNTS>
 __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, uint32_t warp, uint32_t lane,
@@ -55,7 +55,7 @@ __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, ui
 // AVG: Averaging (else Majority Vote).  COUNTS: per-coordinate counts are needed
 // (Averaging, or count_out requested).
 template <int PLANES, bool AVG, bool COUNTS>
-__global__ void __launch_bounds__(kThreads, kMinBlocks)
+__global__ void __launch_bounds__(kThreads, PLANES >= 7 ? 4 : kMinBlocks)
 aggregate_apply_kernel(const __grid_constant__ AggParams p) {
     // Delta of Averaging for every count P, one private copy per warp: it is
     // filled after the tile's first loads are in flight and needs no block barrier.

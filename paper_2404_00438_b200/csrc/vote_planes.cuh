@@ -41,8 +41,8 @@ __device__ __forceinline__ void add8(uint32_t (&pl)[kMaxPlanes], const uint32_t*
 }
 
 // Adds the n workers' words of one word position (col, col + w_stride, ...).
-// Whole groups of 16 workers are fetched with 16 loads issued before the adders
-// run; what is left (fewer than 16) goes in ONE more batch of 8 or 16 guarded
+// Whole groups of 16 workers (32 once N >= 64) are fetched with all their loads
+// issued before the adders run; what is left (fewer than 16) goes in ONE more batch of 8 or 16 guarded
 // loads, slots past the last worker adding zero.  So N <= 16 costs one round trip
 // to memory and every further 16 workers one more.
 // live = false reads nothing at all (the word position holds no parameter).
@@ -53,6 +53,19 @@ __device__ __forceinline__ void count_votes(uint32_t (&pl)[kMaxPlanes], const ui
     for (int p = 0; p < kMaxPlanes; ++p) pl[p] = 0;
     if (!live) return;
     uint32_t i = 0;
+    if constexpr (PLANES >= 7) {
+        // N >= 64: the votes outweigh x; 32 words per round trip (the kernel then
+        // runs with a larger register budget and fewer blocks per SM)
+        for (; i + 32 <= n; i += 32) {
+            uint32_t w[32];
+#pragma unroll
+            for (int q = 0; q < 32; ++q) w[q] = __ldg(col + (i + q) * w_stride);
+            add8<PLANES>(pl, w);
+            add8<PLANES>(pl, w + 8);
+            add8<PLANES>(pl, w + 16);
+            add8<PLANES>(pl, w + 24);
+        }
+    }
     if constexpr (PLANES >= 5) {
         for (; i + 16 <= n; i += 16) {
             uint32_t w[16];
