@@ -287,3 +287,26 @@ def test_new_setters_reject_bad_arguments(dl):
         ctx.set_momentum_dtype(7)
     assert e.value.status == dl.EINVAL
     ctx.destroy()
+
+
+# ---------------------------------------------------------------- seeded random configurations
+@pytest.mark.parametrize("seed", range(24))
+def test_random_configurations(dl, seed):
+    """Random segment tables (empty, tiny, ragged, multi-tile tensors), N, aggregation rule,
+    gradient type and hyper-parameters; every path against the oracle."""
+    rng = np.random.default_rng(1000 + seed)
+    nseg = int(rng.integers(1, 9))
+    numels = [int(rng.choice([0, 1, 31, 33, 127, 129, 4095, 4096, 4097,
+                              int(rng.integers(1, 20000)), int(rng.integers(1, 3 * 4096 * 4))]))
+              for _ in range(nseg)]
+    n = int(rng.choice([1, 2, 3, 4, 6, 8, 9, 15, 16, 17, 31, 32, 33, 63, 64, 65, 100, 200, 255]))
+    mode = int(rng.integers(0, 2))
+    gd = str(rng.choice(["f32", "bf16"]))
+    w = inputs.custom(numels, n, mode, gd, scale=1.0 if gd == "f32" else 1e-3,
+                      a_private=float(rng.choice([0.25, 0.5, 1.0, 2.0])),
+                      beta1=float(rng.choice([0.0, 0.5, 0.9, 0.95, 1.0])),
+                      beta2=float(rng.choice([0.0, 0.75, 0.99, 0.999, 1.0])),
+                      lr=float(rng.choice([1e-4, 1e-2, 0.25])), weight_decay=float(rng.choice([0.0, 0.1, 1.0, 10.0])),
+                      zero_frac=float(rng.choice([0.0, 0.05])), seed=int(rng.integers(0, 1 << 30)))
+    for path in ("two_stage", "fused") + (("per_worker",) if n <= 9 else ()):
+        assert gp.run_small(dl, w, 3, path, modes=(mode,)) == 0
