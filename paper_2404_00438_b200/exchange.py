@@ -1,0 +1,114 @@
+"""Distributed Lion with one worker per process (one process per GPU).
+
+The deployment the paper describes (Algorithm 1; Section 3.2 "Communication
+Cost"): every worker keeps its own momentum, sends only its binary update to
+the server, and receives the aggregated update back.  Here the server's work is
+spread over the workers, the 1-bit analogue of reduce-scatter + all-gather:
+
+  1. worker side, local             delta_r = sign(...), m_r <- ...      (d bits out)
+  2. all-to-all of bit shards       rank r receives coordinate slice r of every worker
+  3. vote on the slice, local       the broadcast message for slice r (1 or K bit planes)
+  4. all-gather of the message      every rank now holds Delta for all d coordinates
+  5. apply, local                   x <- x - eps (Delta + lambda x)
+
+Per rank and step this moves d*(world-1)/world/8 bytes out in step 2 and
+K*d*(world-1)/world/8 bytes in step 4 (K = 1 for Majority Vote,
+ceil(log2(N+1)) for Averaging): Table 1 of the paper, against 4d bytes each way
+for an fp32 gradient exchange.
+
+Steps 1, 3 and 5 are three calls of the C ABI (``dlion_worker_step``,
+``dlion_aggregate``, ``dlion_apply_delta``); steps 2 and 4 are
+``torch.distributed`` collectives (NCCL on GPUs).  Received shards land in this
+rank's own memory and are read with ordinary loads.  This module only
+orchestrates; it holds no optimizer arithmetic.  The three local steps are
+reached through a small ``kernels`` object so that the orchestration can be
+exercised on CPU ranks (``gloo``) with a stand-in for the CUDA library.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+import torch.distributed as dist
+
+ALIGN = 128
+
+
+def padded_length(d_pad: int, world: int) -> int:
+    """Arena length that splits into ``world`` equal slices of whole 128-coordinate groups."""
+    q = ALIGN * world
+    return (d_pad + q - 1) // q * q
+
+
+def planes(n_workers: int, mode: int) -> int:
+    """Bit planes of the broadcast message: 1 (Majority Vote) or ceil(log2(N+1)) (Averaging)."""
+    return 1 if mode == 0 else max(1, n_workers.bit_length())
+
+
+class DlionKernels:
+    """The three local steps on this rank's GPU through the CUDA library."""
+
+    def __init__(self, segments, d_pad_x: int, world: int, rank: int, beta1: float, beta2: float,
+                 lr: float, weight_decay: float, mode: int, gdtype: int):
+        from . import dlion
+        slice_len = d_pad_x // world
+        # this rank as a worker: one worker's state over the whole model
+        self.worker = dlion.Dlion(segments, d_pad_x, 1, beta1, beta2, lr, weight_decay, mode, gdtype)
+        # this rank as the server of its slice: all workers' bits for slice_len coordinates
+        self.server = dlion.Dlion([(0, slice_len)], slice_len, world, beta1, beta2, lr, weight_decay,
+                                  mode, gdtype)
+        # every rank applies the broadcast update to its copy of x
+        self.applier = dlion.Dlion(segments, d_pad_x, world, beta1, beta2, lr, weight_decay, mode, gdtype)
+
+    def set_lr(self, lr: float) -> None:
+        self.applier.set_lr(lr)
+
+    def worker_step(self, g: torch.Tensor, m: torch.Tensor, packed: torch.Tensor) -> None:
+        self.worker.worker_step(0, g, m, packed)
+
+    def aggregate(self, packed_slices: torch.Tensor, wire_slice: torch.Tensor) -> None:
+        self.server.aggregate(packed_slices, wire_slice)
+
+    def apply_delta(self, wire: torch.Tensor, x: torch.Tensor) -> None:
+        self.applier.apply_delta(wire, x)
+
+
+class DistributedLion:
+    """One rank of Distributed Lion.  ``g``, ``m``, ``x`` have ``d_pad_x`` elements
+    (``padded_length(d_pad, world)``); ``m`` is this worker's own momentum."""
+
+    def __init__(self, segments: Sequence[Tuple[int, int]], d_pad: int, mode: int, kernels=None,
+                 beta1: float = 0.9, beta2: float = 0.99, lr: float = 1e-4, weight_decay: float = 0.0,
+                 gdtype: int = 0, group: Optional[dist.ProcessGroup] = None,
+                 device: Optional[torch.device] = None):
+        self.group = group
+        self.world = dist.get_world_size(group)
+        self.rank = dist.get_rank(group)
+        self.mode = mode
+        self.d_pad_x = padded_length(d_pad, self.world)
+        self.words = self.d_pad_x // 32
+        self.slice_words = self.words // self.world
+        self.k = planes(self.world, mode)
+        self.kernels = kernels if kernels is not None else DlionKernels(
+            segments, self.d_pad_x, self.world, self.rank, beta1, beta2, lr, weight_decay, mode, gdtype)
+        dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+        z = dict(dtype=torch.int32, device=dev)
+        self.packed = torch.zeros(self.words, **z)                           # my delta, all coordinates
+        self.recv = torch.zeros(self.world, self.slice_words, **z)           # everyone's delta, my slice
+        self.wire_slice = torch.zeros(self.k, self.slice_words, **z)         # message for my slice
+        self.gathered = torch.zeros(self.world, self.k, self.slice_words, **z)
+        self.wire = torch.zeros(self.k, self.words, **z)                     # message, all coordinates
+
+    def wire_bytes_per_step(self) -> Tuple[int, int]:
+        """(bytes this rank sends in the all-to-all, bytes it receives in the all-gather)."""
+        others = self.world - 1
+        return others * self.slice_words * 4, others * self.k * self.slice_words * 4
+
+    def step(self, g: torch.Tensor, m: torch.Tensor, x: torch.Tensor) -> None:
+        self.kernels.worker_step(g, m, self.packed)
+        dist.all_to_all_single(self.recv.view(-1), self.packed, group=self.group)
+        self.kernels.aggregate(self.recv, self.wire_slice)
+        dist.all_gather_into_tensor(self.gathered.view(-1), self.wire_slice.view(-1), group=self.group)
+        # [rank][plane][slice word] -> [plane][rank][slice word] = plane-major over all coordinates
+        self.wire.view(self.k, self.world, self.slice_words).copy_(self.gathered.permute(1, 0, 2))
+        self.kernels.apply_delta(self.wire, x)

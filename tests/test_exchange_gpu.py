@@ -1,0 +1,50 @@
+"""The exchange path on one GPU: a one-rank NCCL group drives DlionKernels (the three C-ABI
+calls) and the two collectives end to end; the result must equal the single-process step and
+the oracle.  (More than one GPU is not available to these tests; the multi-rank layout is
+covered on CPU ranks in test_exchange_gloo.py.)"""
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+
+from paper_2404_00438_b200 import exchange, inputs
+from tests import gpu_parity as gp
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("mode", [inputs.MAJORITY, inputs.AVERAGE])
+def test_single_rank_exchange_matches_oracle(mode):
+    assert torch.cuda.is_available()
+    from paper_2404_00438_b200 import build
+    build.build()
+    from oracle import dlion_oracle as orc
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
+    try:
+        w = inputs.custom([70000, 333, 4097], 1, mode, "bf16", scale=1e-3, lr=1e-3, weight_decay=1.0)
+        opt = exchange.DistributedLion(w.segments, w.d_pad, mode, beta1=w.beta1, beta2=w.beta2, lr=w.lr,
+                                       weight_decay=w.weight_decay, gdtype=1)
+        D = opt.d_pad_x
+        assert D == w.d_pad
+        x0 = inputs.fill_x0(w, torch.empty(D))
+        x, m = x0.to(dev), torch.zeros(D, device=dev)
+        x_ref, m_ref = x0.numpy().copy(), np.zeros((1, D), np.float32)
+        for t in range(3):
+            g = inputs.fill_grads(w, t, torch.empty(1, D, dtype=torch.bfloat16))
+            opt.step(g[0].to(dev), m, x)
+            torch.cuda.synchronize()
+            packed = np.zeros((1, D // 32), np.uint32)
+            orc.worker_step(w.segments, D, 1, inputs.as_numpy_grads(g), m_ref, packed, w.beta1, w.beta2)
+            orc.aggregate_apply(w.segments, D, 1, mode, packed, x_ref, w.lr, w.weight_decay)
+            gp.compare("packed", opt.packed.cpu().numpy().view(np.uint32), packed[0], True)
+            assert gp.compare("m", m.cpu().numpy(), m_ref[0], False) == 0
+            assert gp.compare("x", x.cpu().numpy(), x_ref, False) == 0
+    finally:
+        dist.destroy_process_group()
