@@ -125,6 +125,30 @@ class ClockSampler:
         return out
 
 
+def host_memory_available() -> int:
+    """Bytes of host memory this process may still take (the tighter of the machine's and the cgroup's)."""
+    try:
+        import psutil
+        avail = int(psutil.virtual_memory().available)
+    except Exception:
+        avail = 1 << 62
+    for path in ("/sys/fs/cgroup/memory.max", "/sys/fs/cgroup/memory/memory.limit_in_bytes"):
+        try:
+            v = open(path).read().strip()
+            if v.isdigit():
+                used = 0
+                for up in ("/sys/fs/cgroup/memory.current", "/sys/fs/cgroup/memory/memory.usage_in_bytes"):
+                    try:
+                        used = int(open(up).read().strip())
+                        break
+                    except Exception:
+                        pass
+                avail = min(avail, int(v) - used)
+        except Exception:
+            pass
+    return avail
+
+
 def bytes_per_param_worker_k1(w, state_bytes: int = 4) -> float:
     """Worker-side kernel: gradient + momentum read + momentum write + 1/8 B of signs."""
     return w.grad_bytes + 2 * state_bytes + 1 / 8
@@ -310,7 +334,12 @@ def run_ours(args):
     # ---- end to end: gradients in pinned host memory, Delta read back
     e2e = None
     if not args.no_e2e:
-        e2e = run_e2e(args, ctx, w, mode, g, m, x, packed, dev, world, barrier)
+        need = N * D * w.grad_bytes * int(os.environ.get("LOCAL_WORLD_SIZE", world))
+        if host_memory_available() >= 1.25 * need:            # every local rank pins its own gradient copy
+            e2e = run_e2e(args, ctx, w, mode, g, m, x, packed, dev, world, barrier)
+        else:
+            e2e = {"value": None, "unit": UNIT, "skipped": "not enough host memory to pin the gradients of every rank",
+                   "h2d_bytes_per_step": N * D * w.grad_bytes, "d2h_bytes_per_step": None}
 
     if rank == 0:
         peak, peak_src = measured_peak()
