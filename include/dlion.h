@@ -38,7 +38,8 @@
  *
  * Calls that launch work are asynchronous on the given CUDA stream (a
  * cudaStream_t passed as void*; NULL = the default stream) and never
- * synchronise.  The context's device must be current.  Nothing here throws,
+ * synchronise.  The context's device must be current.  A context is not
+ * thread-safe: serialise calls on one context.  Nothing here throws,
  * aborts or traps: every failure is a status code.  No CPU fallback exists.
  */
 #ifndef DLION_H_
