@@ -112,3 +112,56 @@ class DistributedLion:
         # [rank][plane][slice word] -> [plane][rank][slice word] = plane-major over all coordinates
         self.wire.view(self.k, self.world, self.slice_words).copy_(self.gathered.permute(1, 0, 2))
         self.kernels.apply_delta(self.wire, x)
+
+
+class LionOptimizer:
+    """Distributed Lion for a list of fp32 parameters on this rank's device.
+
+    The parameters are moved into one flat fp32 arena (each tensor starts on a
+    128-element boundary) and re-pointed at views of it; their ``.grad`` become views
+    of a second flat arena, so backward() accumulates straight into the buffer the
+    worker-side kernel reads.  ``step()`` is one iteration of Algorithm 1 over all
+    of them: one worker-side launch, the exchange, one apply launch.  With a
+    one-rank group this is plain Lion (Eq. 1 of the paper).
+    """
+
+    def __init__(self, params, lr: float = 1e-4, betas: Tuple[float, float] = (0.9, 0.99),
+                 weight_decay: float = 0.0, mode: int = 0, group: Optional[dist.ProcessGroup] = None,
+                 kernels=None):
+        self.params: List[torch.nn.Parameter] = [p for p in params]
+        if not self.params:
+            raise ValueError("no parameters")
+        dev = self.params[0].device
+        for p in self.params:
+            if p.dtype != torch.float32 or p.device != dev:
+                raise ValueError("parameters must be fp32 and on one device")
+        self.segments, off = [], 0
+        for p in self.params:
+            self.segments.append((off, p.numel()))
+            off += (p.numel() + ALIGN - 1) // ALIGN * ALIGN
+        d_pad = max(off, ALIGN)
+        self.core = DistributedLion(self.segments, d_pad, mode, kernels=kernels, beta1=betas[0], beta2=betas[1],
+                                    lr=lr, weight_decay=weight_decay, gdtype=0, group=group, device=dev)
+        n = self.core.d_pad_x
+        self.x = torch.zeros(n, dtype=torch.float32, device=dev)
+        self.g = torch.zeros(n, dtype=torch.float32, device=dev)
+        self.m = torch.zeros(n, dtype=torch.float32, device=dev)
+        with torch.no_grad():
+            for p, (o, k) in zip(self.params, self.segments):
+                self.x[o:o + k].copy_(p.detach().reshape(-1))
+                p.data = self.x[o:o + k].view(p.shape)
+                p.grad = self.g[o:o + k].view(p.shape)
+
+    def set_lr(self, lr: float) -> None:
+        self.core.kernels.set_lr(lr)
+
+    def zero_grad(self) -> None:
+        self.g.zero_()                      # the views stay bound to the arena
+
+    @torch.no_grad()
+    def step(self) -> None:
+        for p, (o, k) in zip(self.params, self.segments):
+            if p.grad is None or p.grad.data_ptr() != self.g[o:o + k].data_ptr():
+                raise RuntimeError("a parameter's .grad no longer points into the gradient arena "
+                                   "(use this optimizer's zero_grad(), not set_to_none)")
+        self.core.step(self.g, self.m, self.x)

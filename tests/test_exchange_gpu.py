@@ -48,3 +48,43 @@ def test_single_rank_exchange_matches_oracle(mode):
             assert gp.compare("x", x.cpu().numpy(), x_ref, False) == 0
     finally:
         dist.destroy_process_group()
+
+
+def test_optimizer_wrapper_trains_a_small_model_like_the_oracle():
+    """Parameters re-pointed at the flat arena, gradients accumulated by autograd straight into
+    the gradient arena, three steps; the arena must equal the oracle's x on the same gradients."""
+    from paper_2404_00438_b200 import build
+    build.build()
+    from oracle import dlion_oracle as orc
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
+    try:
+        torch.manual_seed(0)
+        model = torch.nn.Sequential(torch.nn.Linear(37, 64), torch.nn.Tanh(), torch.nn.Linear(64, 5)).to(dev)
+        opt = exchange.LionOptimizer(model.parameters(), lr=1e-2, betas=(0.9, 0.99), weight_decay=0.1, mode=0)
+        D = opt.core.d_pad_x
+        x_ref = opt.x.cpu().numpy().copy()
+        m_ref = np.zeros((1, D), np.float32)
+        data = torch.randn(16, 37, device=dev)
+        target = torch.randn(16, 5, device=dev)
+        for t in range(3):
+            opt.zero_grad()
+            loss = torch.nn.functional.mse_loss(model(data), target)
+            loss.backward()
+            g = opt.g.cpu().numpy().reshape(1, D).copy()
+            assert np.abs(g).max() > 0
+            opt.step()
+            torch.cuda.synchronize()
+            packed = np.zeros((1, D // 32), np.uint32)
+            orc.worker_step(opt.segments, D, 1, g, m_ref, packed, 0.9, 0.99)
+            orc.aggregate_apply(opt.segments, D, 1, 0, packed, x_ref, 1e-2, 0.1)
+            assert gp.compare("x", opt.x.cpu().numpy(), x_ref, False) == 0
+            flat = torch.cat([p.detach().reshape(-1) for p in model.parameters()]).cpu().numpy()
+            want = np.concatenate([x_ref[o:o + k] for o, k in opt.segments])
+            assert np.array_equal(flat, want)                   # the model really sees the arena
+    finally:
+        dist.destroy_process_group()
