@@ -310,3 +310,49 @@ def test_random_configurations(dl, seed):
                       zero_frac=float(rng.choice([0.0, 0.05])), seed=int(rng.integers(0, 1 << 30)))
     for path in ("two_stage", "fused") + (("per_worker",) if n <= 9 else ()):
         assert gp.run_small(dl, w, 3, path, modes=(mode,)) == 0
+
+
+# ---------------------------------------------------------------- guard bands
+@pytest.mark.parametrize("gd,state", [("f32", "f32"), ("bf16", "f32"), ("bf16", "bf16")])
+def test_nothing_is_written_outside_the_arenas(dl, gd, state):
+    """Every buffer sits between two sentinel bands; after all kernels have run (full tiles that
+    end exactly at the arena's end, ragged tails, both aggregation rules) the bands are intact."""
+    n = 3
+    w = inputs.custom([4097, 33, 2 * 4096], n, AVG, gd, scale=1.0 if gd == "f32" else 1e-3)
+    dev = torch.device("cuda:0")
+    D, W, G = w.d_pad, w.d_pad // 32, 256                       # G: guard elements on each side
+    gdt = inputs.grad_torch_dtype(w)
+    mdt = torch.bfloat16 if state == "bf16" else torch.float32
+
+    def guarded(numel, dtype, fill):
+        buf = torch.full((numel + 2 * G,), fill, dtype=dtype, device=dev)
+        return buf, buf[G:G + numel]
+
+    gbuf, g = guarded(n * D, gdt, 7.0)
+    mbuf, m = guarded(n * D, mdt, 7.0)
+    xbuf, x = guarded(D, torch.float32, 7.0)
+    pbuf, packed = guarded(n * W, torch.int32, 0x5A5A5A5A)
+    dbuf, dbits = guarded(W, torch.int32, 0x5A5A5A5A)
+    cbuf, count = guarded(D, torch.uint8, 0x5A)
+    g.view(n, D).copy_(inputs.fill_grads(w, 0, torch.empty(n, D, dtype=gdt)))
+    m.zero_(); x.zero_(); packed.zero_(); dbits.zero_(); count.zero_()
+    for mode in (MAJ, AVG):
+        ctx = gp.make_ctx(dl, w, mode)
+        if state == "bf16":
+            ctx.set_momentum_dtype(dl.STATE_BF16)
+        K = ctx.delta_planes()
+        wbuf, wire = guarded(K * W, torch.int32, 0x5A5A5A5A)
+        wire.zero_()
+        ctx.worker_step(-1, g.view(n, D), m.view(n, D), packed.view(n, W))
+        for i in range(n):
+            ctx.worker_step(i, g.view(n, D)[i], m.view(n, D)[i], packed.view(n, W)[i])
+        ctx.aggregate_apply(packed, x, dbits, count)
+        ctx.step_fused(g, m, x, packed)
+        ctx.aggregate(packed, wire)
+        ctx.apply_delta(wire, x)
+        torch.cuda.synchronize()
+        for name, buf, fill in (("g", gbuf, 7.0), ("m", mbuf, 7.0), ("x", xbuf, 7.0), ("packed", pbuf, 0x5A5A5A5A),
+                                ("delta_bits", dbuf, 0x5A5A5A5A), ("count", cbuf, 0x5A), ("wire", wbuf, 0x5A5A5A5A)):
+            lo, hi = buf[:G], buf[-G:]
+            assert bool((lo == fill).all()) and bool((hi == fill).all()), f"{name}: guard band overwritten"
+        ctx.destroy()
