@@ -397,12 +397,12 @@ def run_e2e(args, ctx, w, mode, g, m, x, packed, dev, world, barrier):
     """dlion_step_host: per step, N*D gradient elements host->device, Delta device->host."""
     import torch.distributed as dist
     N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
-    host_g = torch.empty(N, D, dtype=g.dtype).pin_memory()
+    host_g = torch.empty(N, D, dtype=g.dtype, pin_memory=True)
     host_g.copy_(g)
     staging = torch.empty(2, D, dtype=g.dtype, device=dev)
     wire_bytes = D if mode == inputs.AVERAGE else W * 4
     wire = torch.zeros(wire_bytes, dtype=torch.uint8, device=dev)
-    host_wire = torch.zeros(wire_bytes, dtype=torch.uint8).pin_memory()
+    host_wire = torch.zeros(wire_bytes, dtype=torch.uint8, pin_memory=True)
     stream = torch.cuda.current_stream()
     for _ in range(args.e2e_warmup):
         ctx.step_host(host_g, m, x, packed, staging, wire, host_wire)

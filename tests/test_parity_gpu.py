@@ -356,3 +356,36 @@ def test_nothing_is_written_outside_the_arenas(dl, gd, state):
             lo, hi = buf[:G], buf[-G:]
             assert bool((lo == fill).all()) and bool((hi == fill).all()), f"{name}: guard band overwritten"
         ctx.destroy()
+
+
+def test_bf16_momentum_special_values(dl):
+    """bf16 momentum with +-0, +-Inf, NaN, values that round up to Inf and bf16 denormals: same
+    signs as the oracle, same stored bits wherever the result is a number, NaN where it is NaN."""
+    from oracle import dlion_oracle as orc
+    n, d = 2, 4096 + 200
+    w = inputs.custom([d], n, MAJ, "f32", beta1=0.5, beta2=0.75)
+    D, W = w.d_pad, w.d_pad // 32
+    rng = np.random.default_rng(21)
+    sp16 = np.array([0x0000, 0x8000, 0x3F80, 0xBF80, 0x7F80, 0xFF80, 0x7FC0, 0x0001, 0x8001, 0x7F7F, 0xFF7F, 0x0080],
+                    np.uint16)
+    m0 = rng.choice(sp16, size=(n, D)).astype(np.uint16)
+    sp32 = np.array([0.0, -0.0, 1.0, -1.0, np.nan, np.inf, -np.inf, 1e-42, 3.4e38, -3.4e38, 1.0 + 2.0 ** -8], np.float32)
+    g0 = rng.choice(sp32, size=(n, D)).astype(np.float32)
+    m0[:, d:] = 0
+    g0[:, d:] = 0
+    m_ref, p_ref = m0.copy(), np.zeros((n, W), np.uint32)
+    orc.worker_step_ex(w.segments, D, n, g0, m_ref, p_ref, [0.5] * n, [0.75] * n)
+    dev = torch.device("cuda:0")
+    ctx = gp.make_ctx(dl, w)
+    ctx.set_momentum_dtype(dl.STATE_BF16)
+    m = torch.from_numpy(m0.view(np.int16)).to(dev).view(torch.bfloat16)
+    packed = torch.zeros(n, W, dtype=torch.int32, device=dev)
+    ctx.worker_step(-1, torch.from_numpy(g0).to(dev), m, packed)
+    torch.cuda.synchronize()
+    gp.compare("packed", packed.cpu().numpy().view(np.uint32), p_ref, True)
+    got = m.cpu().view(torch.int16).numpy().view(np.uint16)
+    nan_ref = (m_ref & 0x7FFF) > 0x7F80
+    nan_got = (got & 0x7FFF) > 0x7F80
+    assert np.array_equal(nan_ref, nan_got)
+    assert nan_ref.any() and np.array_equal(got[~nan_ref], m_ref[~nan_ref])
+    ctx.destroy()
