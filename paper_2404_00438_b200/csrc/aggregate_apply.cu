@@ -88,7 +88,7 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
         const unsigned long long word_idx = (t.base + warp * kWarpSpan) / 32 + lane;
         float4 xv[8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) xv[c] = __ldcs(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
+        for (int c = 0; c < 8; ++c) xv[c] = *(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
         if (!have_table) fill_table();
         uint32_t pl[kMaxPlanes];
         count_votes<PLANES>(pl, p.packed + word_idx, p.w_stride, n, true);
@@ -103,7 +103,7 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
             v.y = apply_coord(v.y, delta_value<AVG>(dn, cnt4, 1, avg_table), p.lr, p.wd);
             v.z = apply_coord(v.z, delta_value<AVG>(dn, cnt4, 2, avg_table), p.lr, p.wd);
             v.w = apply_coord(v.w, delta_value<AVG>(dn, cnt4, 3, avg_table), p.lr, p.wd);
-            __stcs(reinterpret_cast<float4*>(p.x + xe + c * kChunk), v);
+            *reinterpret_cast<float4*>(p.x + xe + c * kChunk) = v;
             if constexpr (COUNTS) {
                 if (p.count != nullptr) *reinterpret_cast<uint32_t*>(p.count + xe + c * kChunk) = cnt4;
             }

@@ -81,14 +81,15 @@ __device__ __forceinline__ float apply_coord(float x, float delta, float lr, flo
 __device__ __forceinline__ float bf16_lo(uint32_t pair) { return __uint_as_float(pair << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t pair) { return __uint_as_float(pair & 0xFFFF0000u); }
 
-// Four consecutive gradients as floats, from fp32 or bf16 storage.
+// Four consecutive gradients as floats, from fp32 or bf16 storage.  (Plain loads and
+// stores throughout: evict-first streaming hints measured 3 % slower on B200.)
 template <bool BF16>
 __device__ __forceinline__ float4 load_grad4(const void* g, unsigned long long idx) {
     if constexpr (BF16) {
-        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(g) + idx));
+        const uint2 v = *(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(g) + idx));
         return make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
     } else {
-        return __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(g) + idx));
+        return *(reinterpret_cast<const float4*>(static_cast<const float*>(g) + idx));
     }
 }
 
@@ -114,10 +115,10 @@ __device__ __forceinline__ uint32_t f32_to_bf16_rne(float f) { return pack_bf16x
 template <bool MB16>
 __device__ __forceinline__ float4 load_state4(const void* m, unsigned long long idx) {
     if constexpr (MB16) {
-        const uint2 v = __ldcs(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(m) + idx));
+        const uint2 v = *(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(m) + idx));
         return make_float4(bf16_lo(v.x), bf16_hi(v.x), bf16_lo(v.y), bf16_hi(v.y));
     } else {
-        return __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(m) + idx));
+        return *(reinterpret_cast<const float4*>(static_cast<const float*>(m) + idx));
     }
 }
 
@@ -127,9 +128,9 @@ __device__ __forceinline__ void store_state4(void* m, unsigned long long idx, co
         uint2 o;
         o.x = pack_bf16x2_rne(v.x, v.y);
         o.y = pack_bf16x2_rne(v.z, v.w);
-        __stcs(reinterpret_cast<uint2*>(static_cast<uint16_t*>(m) + idx), o);
+        *reinterpret_cast<uint2*>(static_cast<uint16_t*>(m) + idx) = o;
     } else {
-        __stcs(reinterpret_cast<float4*>(static_cast<float*>(m) + idx), v);
+        *reinterpret_cast<float4*>(static_cast<float*>(m) + idx) = v;
     }
 }
 

@@ -38,9 +38,9 @@ struct WorkerRegs {                       // one worker's gradients and momenta 
 #pragma unroll
         for (int u = 0; u < kChunksPerWarp; ++u) {
             if constexpr (BF16) {
-                g[u].v = __ldcs(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.g) + at + u * kChunk));
+                g[u].v = *(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.g) + at + u * kChunk));
             } else {
-                g[u].v = __ldcs(reinterpret_cast<const float4*>(static_cast<const float*>(p.g) + at + u * kChunk));
+                g[u].v = *(reinterpret_cast<const float4*>(static_cast<const float*>(p.g) + at + u * kChunk));
             }
             m[u] = load_state4<MB16>(p.m, at + u * kChunk);
         }
@@ -151,7 +151,7 @@ step_fused_kernel(const __grid_constant__ FusedParams p) {
             float4 xv[kChunksPerWarp];
 #pragma unroll
             for (int u = 0; u < kChunksPerWarp; ++u) {
-                xv[u] = __ldcs(reinterpret_cast<const float4*>(p.x + e0 + u * kChunk));
+                xv[u] = *(reinterpret_cast<const float4*>(p.x + e0 + u * kChunk));
             }
             uint32_t* wire = p.packed == nullptr ? nullptr : p.packed + (t.base + in_tile) / 32;
             WorkerRegs<BF16, MB16> a, b;
@@ -172,7 +172,7 @@ step_fused_kernel(const __grid_constant__ FusedParams p) {
                 v.y = apply_coord(v.y, delta_of<AVG>((cnt[u] >> 8) & 0xFFu, thr, avg_table), p.lr, p.wd);
                 v.z = apply_coord(v.z, delta_of<AVG>((cnt[u] >> 16) & 0xFFu, thr, avg_table), p.lr, p.wd);
                 v.w = apply_coord(v.w, delta_of<AVG>(cnt[u] >> 24, thr, avg_table), p.lr, p.wd);
-                __stcs(reinterpret_cast<float4*>(p.x + e0 + u * kChunk), v);
+                *reinterpret_cast<float4*>(p.x + e0 + u * kChunk) = v;
             }
         } else {
             ragged_tile<BF16, AVG, MB16>(p, t, in_tile, e0, lane, thr, avg_table);

@@ -68,7 +68,7 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
         float4 xv[8];
         if (full) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) xv[c] = __ldcs(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
+            for (int c = 0; c < 8; ++c) xv[c] = *(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
         }
         uint32_t pl[kMaxPlanes];
         uint32_t dword = 0;
@@ -99,7 +99,7 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
                 v.y = apply_coord(v.y, delta_value<AVG>(dn, cnt4, 1, avg_table), p.lr, p.wd);
                 v.z = apply_coord(v.z, delta_value<AVG>(dn, cnt4, 2, avg_table), p.lr, p.wd);
                 v.w = apply_coord(v.w, delta_value<AVG>(dn, cnt4, 3, avg_table), p.lr, p.wd);
-                __stcs(reinterpret_cast<float4*>(p.x + e), v);
+                *reinterpret_cast<float4*>(p.x + e) = v;
             } else {
                 for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
                     p.x[e + q] = apply_coord(p.x[e + q], delta_value<AVG>(dn, cnt4, q, avg_table), p.lr, p.wd);
