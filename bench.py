@@ -37,7 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # (dram__bytes_read.sum + dram__bytes_write.sum), as bytes per param*worker, keyed
 # by the SHA-256 of the kernel's source at capture time: reported only while the
 # source is unchanged.  See profiles/.
-NCU_TRAFFIC = {("worker_step_kernel", "134f9758da01f13d"): 10.0714}   # profiles/worker_step_kernel_c2.md
+NCU_TRAFFIC = {("worker_step_kernel", "e92caa95f78d0733"): 10.0759}   # profiles/worker_step_kernel_c2.md
 
 
 def kernel_hash() -> str:
