@@ -242,11 +242,12 @@ def run_ours(args):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    from paper_2404_00438_b200 import build, dlion
+    from paper_2404_00438_b200 import build
     if rank == 0:
-        build.build()
+        build.build()                                 # in-tree; a no-op when the library is up to date
     if world > 1:
         dist.barrier()
+    from paper_2404_00438_b200 import dlion           # loads libdlion.so; raises if it is missing
 
     w = inputs.workload(args.workload)
     if args.n_workers:
