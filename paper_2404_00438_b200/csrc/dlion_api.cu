@@ -7,14 +7,13 @@
 #include <vector>
 
 #include "dlion_ctx.cuh"
+#include "host_checks.h"
 
 namespace {
 
-bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
-
-bool unit_interval(float v) { return v >= 0.0f && v <= 1.0f; }           // false for NaN
-
-bool nonneg_finite(float v) { return v >= 0.0f && std::isfinite(v); }
+using dlion::aligned;
+using dlion::nonneg_finite;
+using dlion::unit_interval;
 
 dlion::Betas betas_of(const dlion_ctx* c) {
     dlion::Betas k;

@@ -1,9 +1,10 @@
 // Host-gradient step, analytic wire volume, and context teardown (include/dlion.h).
 #include "dlion_ctx.cuh"
+#include "host_checks.h"
 
 namespace {
 
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) % 16) == 0; }
+using dlion::aligned16;
 
 // Streams and events of the copy pipeline; created once, on first use.
 cudaError_t ensure_pipeline(dlion_ctx* c) {

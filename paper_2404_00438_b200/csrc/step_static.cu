@@ -15,6 +15,7 @@
 #include <mutex>
 
 #include "dlion_common.cuh"
+#include "host_checks.h"
 
 namespace {
 
@@ -59,9 +60,9 @@ __global__ void write_flat_row_kernel(dlion::SegDev* row, unsigned long long d) 
     row->first_tile = 0;
 }
 
-bool unit_interval(float v) { return v >= 0.0f && v <= 1.0f; }
-bool nonneg_finite(float v) { return v >= 0.0f && v <= 3.402823466e38f; }
-bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) % 16) == 0; }
+using dlion::aligned16;
+using dlion::nonneg_finite;
+using dlion::unit_interval;
 
 }  // namespace
 
