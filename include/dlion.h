@@ -53,7 +53,8 @@ extern "C" {
 #endif
 
 #define DLION_ALIGN 128u        /* elements: alignment of segment starts and of d_pad */
-#define DLION_MAX_WORKERS 255u  /* vote counts are kept in 8 bits */
+#define DLION_MAX_WORKERS 65535u /* up to 16 bit planes of votes */
+#define DLION_MAX_WORKERS_BYTE_COUNTS 255u /* count_out, dlion_step_fused, dlion_step_host, dlion_step_static */
 #define DLION_STATIC_MAX_COORD_WORKERS 134217728ull /* dlion_step_static: limit on N * d_pad */
 
 typedef struct dlion_ctx dlion_ctx; /* opaque; host-side object */
@@ -126,7 +127,9 @@ dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, vo
  *   delta_bits_out  out, nullable  [d_pad/32]: bit = (S >= 0), i.e. Delta of
  *                   Majority Vote, the d-bit server->worker message of Table 1
  *   count_out       out, nullable  [d_pad] bytes: P, the integer in {0..N} that
- *                   Averaging sends back (Section 3.2 "Communication Cost") */
+ *                   Averaging sends back (Section 3.2 "Communication Cost");
+ *                   N <= 255 only (DLION_EINVAL otherwise; dlion_aggregate has
+ *                   the bit-plane form for any N) */
 dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float* x,
                                    uint32_t* delta_bits_out, uint8_t* count_out,
                                    void* cuda_stream);
@@ -161,6 +164,7 @@ uint32_t dlion_delta_planes(const dlion_ctx* ctx);
 /* The whole of one Algorithm-1 iteration in ONE launch: a thread block holds a
  * tile of coordinates for all N workers, votes in registers and applies x.
  * Same results as dlion_worker_step(-1) followed by dlion_aggregate_apply.
+ * N <= 255 (votes are counted in bytes); DLION_EINVAL beyond.
  *   packed_out  out, nullable: the wire buffer, if the caller still wants it. */
 dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float* x,
                               uint32_t* packed_out, void* cuda_stream);
@@ -191,7 +195,7 @@ dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, void* m, fl
  * handed.  The segment table and the 1-bit wire buffer live in a fixed array
  * inside the library image (16 MiB + 256 B per GPU that loads the library, held
  * until the process exits).  The call allocates nothing, on host or device.
- *   d, n_workers   the problem; d_pad = d rounded up to DLION_ALIGN, and
+ *   d, n_workers   the problem (n_workers <= 255); d_pad = d rounded up to DLION_ALIGN, and
  *                  n_workers * d_pad <= DLION_STATIC_MAX_COORD_WORKERS, else
  *                  DLION_EINVAL ("does not fit the fixed scratch")
  *   grads [N][d_pad], m [N][d_pad] (in/out), x [d_pad] (in/out): device, 16-byte

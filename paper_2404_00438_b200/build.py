@@ -14,6 +14,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB = os.path.join(_HERE, "libdlion.so")
+OBJDIR = os.path.join(_HERE, "_build")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -43,14 +44,28 @@ def is_stale() -> bool:
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Build ``libdlion.so`` if it is missing or older than its sources."""
+    """Build ``libdlion.so`` if it is missing or older than its sources.
+
+    Each ``.cu`` file is compiled to an object in ``_build/`` (in parallel), then linked.
+    """
     if not force and not is_stale():
         return LIB
-    cmd = [_nvcc(), *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-o", LIB, *sources()]
+    from concurrent.futures import ThreadPoolExecutor
+    nvcc = _nvcc()
+    os.makedirs(OBJDIR, exist_ok=True)
+    compile_flags = [f for f in NVCC_FLAGS if f not in ("-shared", "-cudart", "static")]
     if verbose:
-        cmd.insert(1, "-Xptxas")
-        cmd.insert(2, "-v")
-    subprocess.run(cmd, check=True)
+        compile_flags += ["-Xptxas", "-v"]
+
+    def one(src: str) -> str:
+        obj = os.path.join(OBJDIR, os.path.splitext(os.path.basename(src))[0] + ".o")
+        subprocess.run([nvcc, *compile_flags, "-I", INCLUDE, "-I", CSRC, "-c", "-o", obj, src], check=True)
+        return obj
+
+    with ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as pool:
+        objs = list(pool.map(one, sources()))
+    subprocess.run([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared", "-cudart", "static",
+                    "-o", LIB, *objs], check=True)
     return LIB
 
 

@@ -41,13 +41,12 @@ __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, ui
     if (p.delta_bits != nullptr && nbits != 0) p.delta_bits[word_idx] = dword;
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
-        uint32_t dn, cnt4;
-        my_votes<PLANES, COUNTS>(pl, dword, c, lane, dn, cnt4);
+        const Votes4 v = my_votes<PLANES, COUNTS>(pl, dword, c, lane);
         const uint32_t j0 = w0 + c * kChunk + lane * 4;
         const unsigned long long e = t.base + j0;
         for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
-            p.x[e + q] = apply_coord(p.x[e + q], delta_value<AVG>(dn, cnt4, q, avg_table), p.lr, p.wd);
-            if (p.count != nullptr) p.count[e + q] = static_cast<uint8_t>((cnt4 >> (8 * q)) & 0xFFu);
+            p.x[e + q] = apply_coord(p.x[e + q], delta_value<PLANES, AVG>(v, q, avg_table, p.n_workers), p.lr, p.wd);
+            if (p.count != nullptr) p.count[e + q] = static_cast<uint8_t>(count_of<PLANES>(v, q));
         }
     }
 }
@@ -59,19 +58,15 @@ __global__ void __launch_bounds__(kThreads, PLANES >= 7 ? 4 : kMinBlocks)
 aggregate_apply_kernel(const __grid_constant__ AggParams p) {
     // Delta of Averaging for every count P, one private copy per warp: it is
     // filled after the tile's first loads are in flight and needs no block barrier.
-    __shared__ float avg_tables[AVG ? kThreads / 32 : 1][AVG ? 256 : 1];
+    __shared__ float avg_tables[(AVG && PLANES <= 8) ? kThreads / 32 : 1][(AVG && PLANES <= 8) ? 256 : 1];
     const uint32_t n = p.n_workers;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t thr = (n + 1u) >> 1;   // 2P >= N  <=>  P >= ceil(N/2)
-    float* avg_table = avg_tables[AVG ? warp : 0];
+    float* avg_table = avg_tables[(AVG && PLANES <= 8) ? warp : 0];
     bool have_table = !AVG;
     auto fill_table = [&]() {
-        for (uint32_t c = lane; c <= n; c += 32) {
-            avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
-                                     static_cast<float>(n));
-        }
-        __syncwarp();
+        fill_avg_table<PLANES>(avg_table, n, lane);
         have_table = true;
     };
 
@@ -96,16 +91,15 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
         if (p.delta_bits != nullptr) p.delta_bits[word_idx] = dword;
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            uint32_t dn, cnt4;
-            my_votes<PLANES, COUNTS>(pl, dword, c, lane, dn, cnt4);
+            const Votes4 vt = my_votes<PLANES, COUNTS>(pl, dword, c, lane);
             float4 v = xv[c];
-            v.x = apply_coord(v.x, delta_value<AVG>(dn, cnt4, 0, avg_table), p.lr, p.wd);
-            v.y = apply_coord(v.y, delta_value<AVG>(dn, cnt4, 1, avg_table), p.lr, p.wd);
-            v.z = apply_coord(v.z, delta_value<AVG>(dn, cnt4, 2, avg_table), p.lr, p.wd);
-            v.w = apply_coord(v.w, delta_value<AVG>(dn, cnt4, 3, avg_table), p.lr, p.wd);
+            v.x = apply_coord(v.x, delta_value<PLANES, AVG>(vt, 0, avg_table, n), p.lr, p.wd);
+            v.y = apply_coord(v.y, delta_value<PLANES, AVG>(vt, 1, avg_table, n), p.lr, p.wd);
+            v.z = apply_coord(v.z, delta_value<PLANES, AVG>(vt, 2, avg_table, n), p.lr, p.wd);
+            v.w = apply_coord(v.w, delta_value<PLANES, AVG>(vt, 3, avg_table, n), p.lr, p.wd);
             *reinterpret_cast<float4*>(p.x + xe + c * kChunk) = v;
             if constexpr (COUNTS) {
-                if (p.count != nullptr) *reinterpret_cast<uint32_t*>(p.count + xe + c * kChunk) = cnt4;
+                if (p.count != nullptr) *reinterpret_cast<uint32_t*>(p.count + xe + c * kChunk) = vt.lo;   // N <= 255 here
             }
         }
     }
@@ -129,15 +123,24 @@ cudaError_t launch(const AggParams& p, cudaStream_t s) {
 
 cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s) {
     (void)sm_count;
-    const uint32_t n = p.n_workers;       // planes = bit length of N
-    if (n < 2) return launch<1>(p, s);
-    if (n < 4) return launch<2>(p, s);
-    if (n < 8) return launch<3>(p, s);
-    if (n < 16) return launch<4>(p, s);
-    if (n < 32) return launch<5>(p, s);
-    if (n < 64) return launch<6>(p, s);
-    if (n < 128) return launch<7>(p, s);
-    return launch<8>(p, s);
+    switch (planes_for(p.n_workers)) {    // planes = bit length of N
+        case 1: return launch<1>(p, s);
+        case 2: return launch<2>(p, s);
+        case 3: return launch<3>(p, s);
+        case 4: return launch<4>(p, s);
+        case 5: return launch<5>(p, s);
+        case 6: return launch<6>(p, s);
+        case 7: return launch<7>(p, s);
+        case 8: return launch<8>(p, s);
+        case 9: return launch<9>(p, s);
+        case 10: return launch<10>(p, s);
+        case 11: return launch<11>(p, s);
+        case 12: return launch<12>(p, s);
+        case 13: return launch<13>(p, s);
+        case 14: return launch<14>(p, s);
+        case 15: return launch<15>(p, s);
+        default: return launch<16>(p, s);
+    }
 }
 
 }  // namespace dlion

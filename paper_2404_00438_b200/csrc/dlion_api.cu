@@ -213,6 +213,7 @@ dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, vo
 dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float* x,
                                    uint32_t* delta_bits_out, uint8_t* count_out, void* cuda_stream) {
     if (ctx == nullptr || packed == nullptr || x == nullptr) return DLION_EINVAL;
+    if (count_out != nullptr && ctx->n_workers > DLION_MAX_WORKERS_BYTE_COUNTS) return DLION_EINVAL;
     if (!aligned(packed, 16) || !aligned(x, 16) || !aligned(delta_bits_out, 16) || !aligned(count_out, 4)) {
         return DLION_EALIGN;
     }
@@ -241,6 +242,7 @@ dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float
 dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float* x,
                               uint32_t* packed_out, void* cuda_stream) {
     if (ctx == nullptr || grads == nullptr || m == nullptr || x == nullptr) return DLION_EINVAL;
+    if (ctx->n_workers > DLION_MAX_WORKERS_BYTE_COUNTS) return DLION_EINVAL;       // byte-wide vote counters
     if (!aligned(grads, 16) || !aligned(m, 16) || !aligned(x, 16) || !aligned(packed_out, 16)) {
         return DLION_EALIGN;
     }

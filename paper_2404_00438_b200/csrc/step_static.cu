@@ -71,7 +71,7 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
                                           dlion_gdtype gdtype, const void* grads, float* m, float* x,
                                           void* cuda_stream) {
     if (d == 0 || grads == nullptr || m == nullptr || x == nullptr) return DLION_EINVAL;
-    if (n_workers == 0 || n_workers > DLION_MAX_WORKERS) return DLION_EINVAL;
+    if (n_workers == 0 || n_workers > DLION_MAX_WORKERS_BYTE_COUNTS) return DLION_EINVAL;
     if (!unit_interval(beta1) || !unit_interval(beta2)) return DLION_EINVAL;
     if (!nonneg_finite(lr) || !nonneg_finite(weight_decay)) return DLION_EINVAL;
     if (mode != DLION_MAJORITY && mode != DLION_AVERAGE) return DLION_EINVAL;

@@ -7,7 +7,7 @@
 namespace dlion {
 
 constexpr uint32_t kWarpSpan = 1024;
-constexpr int kMaxPlanes = 8;             // N <= 255
+constexpr int kMaxPlanes = 16;            // N <= 65535
 
 __device__ __forceinline__ void csa(uint32_t& sum, uint32_t& carry, uint32_t a, uint32_t b, uint32_t c) {
     sum = a ^ b ^ c;
@@ -103,27 +103,65 @@ __device__ __forceinline__ uint32_t planes_ge(const uint32_t (&pl)[kMaxPlanes], 
     return gt | eq;
 }
 
-// Delta of my four coordinates in chunk c, and (when counts are needed) their
-// four vote counts, one per byte.  All 32 lanes must call this together.
+// Votes of my four coordinates in chunk c: the Delta bits (dn, bit q = coordinate q)
+// and, when counts are needed, the four vote counts.  Up to 8 planes the counts are
+// packed one per byte in lo; beyond (N > 255) two 16-bit counts each in lo and hi.
+struct Votes4 {
+    uint32_t dn, lo, hi;
+};
+
+// All 32 lanes must call this together.
 template <int PLANES, bool COUNTS>
-__device__ __forceinline__ void my_votes(const uint32_t (&pl)[kMaxPlanes], uint32_t dword, int c, uint32_t lane,
-                                         uint32_t& dn, uint32_t& cnt4) {
+__device__ __forceinline__ Votes4 my_votes(const uint32_t (&pl)[kMaxPlanes], uint32_t dword, int c, uint32_t lane) {
     const uint32_t src = 4u * c + (lane >> 3);           // lane that owns my word
     const uint32_t sh = 4u * (lane & 7u);
-    dn = (__shfl_sync(kFull, dword, src) >> sh) & 0xFu;
-    cnt4 = 0;
+    Votes4 v;
+    v.dn = (__shfl_sync(kFull, dword, src) >> sh) & 0xFu;
+    v.lo = 0;
+    v.hi = 0;
     if constexpr (COUNTS) {
 #pragma unroll
         for (int q = 0; q < PLANES; ++q) {
-            cnt4 += spread_nibble((__shfl_sync(kFull, pl[q], src) >> sh) & 0xFu) << q;
+            const uint32_t nib = (__shfl_sync(kFull, pl[q], src) >> sh) & 0xFu;
+            if constexpr (PLANES <= 8) {
+                v.lo += spread_nibble(nib) << q;
+            } else {
+                v.lo += ((nib & 1u) | ((nib & 2u) << 15)) << q;
+                v.hi += (((nib >> 2) & 1u) | ((nib & 8u) << 13)) << q;
+            }
         }
     }
+    return v;
 }
 
-template <bool AVG>
-__device__ __forceinline__ float delta_value(uint32_t dn, uint32_t cnt4, int q, const float* avg_table) {
-    if constexpr (AVG) return avg_table[(cnt4 >> (8 * q)) & 0xFFu];
-    return ((dn >> q) & 1u) ? 1.0f : -1.0f;
+template <int PLANES>
+__device__ __forceinline__ uint32_t count_of(const Votes4& v, int q) {
+    if constexpr (PLANES <= 8) return (v.lo >> (8 * q)) & 0xFFu;
+    return ((q < 2 ? v.lo : v.hi) >> (16 * (q & 1))) & 0xFFFFu;
+}
+
+// Delta of coordinate q.  Averaging: from the per-warp table while the counts fit
+// it (N <= 255), else the correctly rounded quotient directly.
+template <int PLANES, bool AVG>
+__device__ __forceinline__ float delta_value(const Votes4& v, int q, const float* avg_table, uint32_t n) {
+    if constexpr (AVG) {
+        const uint32_t c = count_of<PLANES>(v, q);
+        if constexpr (PLANES <= 8) return avg_table[c];
+        return __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)), static_cast<float>(n));
+    }
+    return ((v.dn >> q) & 1u) ? 1.0f : -1.0f;
+}
+
+// Fills a warp's private table of Averaging's Delta for every count (N <= 255 only).
+template <int PLANES>
+__device__ __forceinline__ void fill_avg_table(float* avg_table, uint32_t n, uint32_t lane) {
+    if constexpr (PLANES <= 8) {
+        for (uint32_t c = lane; c <= n; c += 32) {
+            avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
+                                     static_cast<float>(n));
+        }
+        __syncwarp();
+    }
 }
 
 }  // namespace dlion

@@ -49,11 +49,11 @@ aggregate_kernel(const __grid_constant__ WireParams p) {
 template <int PLANES, bool AVG>
 __global__ void __launch_bounds__(kThreads, 6)
 apply_delta_kernel(const __grid_constant__ WireParams p) {
-    __shared__ float avg_tables[AVG ? kThreads / 32 : 1][AVG ? 256 : 1];
+    __shared__ float avg_tables[(AVG && PLANES <= 8) ? kThreads / 32 : 1][(AVG && PLANES <= 8) ? 256 : 1];
     const uint32_t n = p.n_workers;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
-    float* avg_table = avg_tables[AVG ? warp : 0];
+    float* avg_table = avg_tables[(AVG && PLANES <= 8) ? warp : 0];
     bool have_table = !AVG;
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
@@ -79,30 +79,25 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
             dword = live ? __ldg(p.wire_in + word_idx) : 0u;
         }
         if (!have_table) {
-            for (uint32_t c = lane; c <= n; c += 32) {
-                avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
-                                         static_cast<float>(n));
-            }
-            __syncwarp();
+            fill_avg_table<PLANES>(avg_table, n, lane);
             have_table = true;
         }
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            uint32_t dn, cnt4;
-            my_votes<PLANES, AVG>(pl, dword, c, lane, dn, cnt4);
+            const Votes4 vt = my_votes<PLANES, AVG>(pl, dword, c, lane);
             const uint32_t j0 = w0 + c * kChunk + lane * 4;
             if (j0 >= t.valid) continue;                            // after the shuffles: all lanes took part
             const unsigned long long e = xe + c * kChunk;
             if (full) {
                 float4 v = xv[c];
-                v.x = apply_coord(v.x, delta_value<AVG>(dn, cnt4, 0, avg_table), p.lr, p.wd);
-                v.y = apply_coord(v.y, delta_value<AVG>(dn, cnt4, 1, avg_table), p.lr, p.wd);
-                v.z = apply_coord(v.z, delta_value<AVG>(dn, cnt4, 2, avg_table), p.lr, p.wd);
-                v.w = apply_coord(v.w, delta_value<AVG>(dn, cnt4, 3, avg_table), p.lr, p.wd);
+                v.x = apply_coord(v.x, delta_value<PLANES, AVG>(vt, 0, avg_table, n), p.lr, p.wd);
+                v.y = apply_coord(v.y, delta_value<PLANES, AVG>(vt, 1, avg_table, n), p.lr, p.wd);
+                v.z = apply_coord(v.z, delta_value<PLANES, AVG>(vt, 2, avg_table, n), p.lr, p.wd);
+                v.w = apply_coord(v.w, delta_value<PLANES, AVG>(vt, 3, avg_table, n), p.lr, p.wd);
                 *reinterpret_cast<float4*>(p.x + e) = v;
             } else {
                 for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
-                    p.x[e + q] = apply_coord(p.x[e + q], delta_value<AVG>(dn, cnt4, q, avg_table), p.lr, p.wd);
+                    p.x[e + q] = apply_coord(p.x[e + q], delta_value<PLANES, AVG>(vt, q, avg_table, n), p.lr, p.wd);
                 }
             }
         }
@@ -140,7 +135,15 @@ cudaError_t launch_wire(const WireParams& p, bool apply, cudaStream_t s) {
         case 5: return launch<5>(p, apply, s);
         case 6: return launch<6>(p, apply, s);
         case 7: return launch<7>(p, apply, s);
-        default: return launch<8>(p, apply, s);
+        case 8: return launch<8>(p, apply, s);
+        case 9: return launch<9>(p, apply, s);
+        case 10: return launch<10>(p, apply, s);
+        case 11: return launch<11>(p, apply, s);
+        case 12: return launch<12>(p, apply, s);
+        case 13: return launch<13>(p, apply, s);
+        case 14: return launch<14>(p, apply, s);
+        case 15: return launch<15>(p, apply, s);
+        default: return launch<16>(p, apply, s);
     }
 }
 

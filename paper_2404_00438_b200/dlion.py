@@ -19,7 +19,7 @@ MAJORITY, AVERAGE = 0, 1
 GRAD_F32, GRAD_BF16 = 0, 1
 STATE_F32, STATE_BF16 = 0, 1
 ALIGN = 128
-MAX_WORKERS = 255
+MAX_WORKERS = 65535
 OK, EINVAL, EALIGN, ENOMEM, ECUDA, ESTATE = range(6)
 
 EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_set_momentum_dtype",

@@ -352,7 +352,7 @@ def check_delta_wire_roundtrip(lib):
     for o, n in segs:
         valid[o:o + n] = True
     d = int(valid.sum())
-    for N in (1, 2, 3, 4, 7, 8, 16, 33, 255):
+    for N in (1, 2, 3, 4, 7, 8, 16, 33, 255, 256, 1000):
         bits = (rng.random((N, d_pad)) < rng.random(d_pad)[None, :]) & valid[None, :]
         packed = np.packbits(bits, axis=1, bitorder="little").view(np.uint32).reshape(N, -1).copy()
         P = bits.sum(axis=0).astype(np.int64)

@@ -50,7 +50,7 @@ def test_check_layout(dl):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(n_workers=0), dict(n_workers=256), dict(beta1=-0.1), dict(beta1=1.5), dict(beta2=float("nan")),
+    dict(n_workers=0), dict(n_workers=65536), dict(beta1=-0.1), dict(beta1=1.5), dict(beta2=float("nan")),
     dict(lr=-1.0), dict(lr=float("inf")), dict(weight_decay=-0.5), dict(mode=2), dict(gdtype=7),
 ])
 def test_init_rejects_bad_arguments_before_cuda(dl, kw):

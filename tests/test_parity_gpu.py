@@ -175,7 +175,7 @@ def test_step_host_matches_oracle(dl, mode):
 
 
 # ---------------------------------------------------------------- server-only aggregate + worker-side apply
-@pytest.mark.parametrize("n", [1, 2, 3, 4, 7, 8, 16, 33, 64, 255])
+@pytest.mark.parametrize("n", [1, 2, 3, 4, 7, 8, 16, 33, 64, 255, 256, 300, 1000, 4097])
 @pytest.mark.parametrize("mode", [MAJ, AVG])
 def test_aggregate_then_apply_delta(dl, n, mode):
     from oracle import dlion_oracle as orc
@@ -388,4 +388,24 @@ def test_bf16_momentum_special_values(dl):
     nan_got = (got & 0x7FFF) > 0x7F80
     assert np.array_equal(nan_ref, nan_got)
     assert nan_ref.any() and np.array_equal(got[~nan_ref], m_ref[~nan_ref])
+    ctx.destroy()
+
+
+# ---------------------------------------------------------------- more than 255 workers
+@pytest.mark.parametrize("n", [256, 511, 1000])
+@pytest.mark.parametrize("mode", [MAJ, AVG])
+def test_more_than_255_workers(dl, n, mode):
+    """Vote counts beyond one byte: 9 and 10 bit planes; the byte-count outputs and the fused
+    step say so instead of overflowing."""
+    w = inputs.custom([4096 + 77, 33], n, mode, "bf16", scale=1e-3, lr=1e-3, weight_decay=0.5)
+    assert gp.run_small(dl, w, 2, "two_stage", modes=(mode,)) == 0
+    dev = torch.device("cuda:0")
+    ctx = gp.make_ctx(dl, w)
+    t = torch.zeros(n * w.d_pad, dtype=torch.int32, device=dev)
+    with pytest.raises(dl.DlionError) as e:
+        ctx.step_fused(t.view(torch.bfloat16)[:n * w.d_pad], t.view(torch.float32), t.view(torch.float32)[:w.d_pad], None)
+    assert e.value.status == dl.EINVAL
+    with pytest.raises(dl.DlionError) as e:
+        ctx.aggregate_apply(t, t.view(torch.float32)[:w.d_pad], None, t.view(torch.uint8)[:w.d_pad])
+    assert e.value.status == dl.EINVAL
     ctx.destroy()
