@@ -409,3 +409,36 @@ def test_more_than_255_workers(dl, n, mode):
         ctx.aggregate_apply(t, t.view(torch.float32)[:w.d_pad], None, t.view(torch.uint8)[:w.d_pad])
     assert e.value.status == dl.EINVAL
     ctx.destroy()
+
+
+def test_step_host_with_bf16_momentum_and_worker_betas(dl):
+    """The host-gradient step slices the momentum arena by its storage type and passes each
+    worker's own betas."""
+    from oracle import dlion_oracle as orc
+    n = 3
+    b1s, b2s = [0.9, 0.5, 0.0], [0.99, 0.75, 0.0]
+    w = inputs.custom([9000, 77], n, MAJ, "bf16", scale=1e-3, lr=1e-3, weight_decay=1.0)
+    dev = torch.device("cuda:0")
+    D, W = w.d_pad, w.d_pad // 32
+    ctx = gp.make_ctx(dl, w)
+    ctx.set_momentum_dtype(dl.STATE_BF16)
+    for i in range(n):
+        ctx.set_worker_betas(i, b1s[i], b2s[i])
+    x0 = inputs.fill_x0(w, torch.empty(D))
+    m_ref, x_ref = np.zeros((n, D), np.uint16), x0.numpy().copy()
+    m = torch.zeros(n, D, dtype=torch.bfloat16, device=dev)
+    x = x0.to(dev)
+    packed = torch.zeros(n, W, dtype=torch.int32, device=dev)
+    staging = torch.empty(2, D, dtype=torch.bfloat16, device=dev)
+    host_g = torch.empty(n, D, dtype=torch.bfloat16).pin_memory()
+    for t in range(3):
+        inputs.fill_grads(w, t, host_g)
+        p_ref = np.zeros((n, W), np.uint32)
+        orc.worker_step_ex(w.segments, D, n, inputs.as_numpy_grads(host_g), m_ref, p_ref, b1s, b2s)
+        orc.aggregate_apply(w.segments, D, n, MAJ, p_ref, x_ref, w.lr, w.weight_decay)
+        ctx.step_host(host_g, m, x, packed, staging)
+        torch.cuda.synchronize()
+        gp.compare("packed", packed.cpu().numpy().view(np.uint32), p_ref, True)
+        assert np.array_equal(m.cpu().view(torch.int16).numpy().view(np.uint16), m_ref)
+        assert gp.compare("x", x.cpu().numpy(), x_ref, False) == 0
+    ctx.destroy()
