@@ -54,7 +54,7 @@ extern "C" {
 
 #define DLION_ALIGN 128u        /* elements: alignment of segment starts and of d_pad */
 #define DLION_MAX_WORKERS 65535u /* up to 16 bit planes of votes */
-#define DLION_MAX_WORKERS_BYTE_COUNTS 255u /* count_out, dlion_step_fused, dlion_step_host, dlion_step_static */
+#define DLION_MAX_WORKERS_BYTE_COUNTS 255u /* count_out, dlion_step_fused, dlion_step_static, dlion_step_host with Averaging */
 #define DLION_STATIC_MAX_COORD_WORKERS 134217728ull /* dlion_step_static: limit on N * d_pad */
 
 typedef struct dlion_ctx dlion_ctx; /* opaque; host-side object */
@@ -177,7 +177,7 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float*
  *   m, x, packed    device     as above (packed is used as the wire buffer)
  *   staging         device     2 * d_pad gradient elements (two slices)
  *   delta_wire_dev  device, nullable  [d_pad/32] words (Majority Vote) or
- *                   [d_pad] bytes (Averaging): Delta as the server sends it
+ *                   [d_pad] bytes (Averaging, N <= 255): Delta as the server sends it
  *   host_delta_out  out, host, nullable: copy of delta_wire_dev; needs
  *                   delta_wire_dev.  Complete when cuda_stream's work is.
  * Uses one internal copy stream ordered against cuda_stream by events. */
