@@ -325,6 +325,29 @@ def run_ours(args):
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     clocks = sampler.stop() if rank == 0 else None
 
+    # ---- optional: the same K steps captured once in a CUDA graph and replayed
+    # (small workloads are bound by launch latency; the calls never synchronise)
+    graph_ms = None
+    if args.graph:
+        side = torch.cuda.Stream()
+        gph = torch.cuda.CUDAGraph()
+        side.wait_stream(stream)
+        with torch.cuda.stream(side):
+            step()
+            torch.cuda.synchronize()
+            with torch.cuda.graph(gph, stream=side):
+                for _ in range(args.steps):
+                    step()
+        torch.cuda.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        gph.replay()
+        barrier()
+        g0.record(stream)
+        gph.replay()
+        g1.record(stream)
+        barrier()
+        graph_ms = g0.elapsed_time(g1) / args.steps
+
     t_all = torch.tensor([total_ms], dtype=torch.float64, device=dev)
     if world > 1:
         dist.all_reduce(t_all, op=dist.ReduceOp.MAX)
@@ -381,7 +404,7 @@ def run_ours(args):
                              else "working set comparable to L2: latency-bound case",
                        "timed_region": "K steps back to back in one bracket, on the last generated gradients",
                        "per_rank": "each rank steps its own full-size coordinate slab; no collective"},
-            "ms_per_step_fresh_grads": fresh_ms,
+            "ms_per_step_fresh_grads": fresh_ms, "ms_per_step_graph_replay": graph_ms,
             "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches, "clocks": clocks,
             "wire_bytes_per_step": {"up_all_workers": up, "down_per_worker": down,
@@ -435,6 +458,7 @@ def main():
     ap.add_argument("--mode", default=None, choices=["majority", "average"])
     ap.add_argument("--path", default="two_stage", choices=["two_stage", "fused"])
     ap.add_argument("--state", default="f32", choices=["f32", "bf16"], help="momentum storage")
+    ap.add_argument("--graph", action="store_true", help="also time the K steps replayed from one CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--e2e-warmup", type=int, default=1)

@@ -442,3 +442,43 @@ def test_step_host_with_bf16_momentum_and_worker_betas(dl):
         assert np.array_equal(m.cpu().view(torch.int16).numpy().view(np.uint16), m_ref)
         assert gp.compare("x", x.cpu().numpy(), x_ref, False) == 0
     ctx.destroy()
+
+
+def test_calls_can_be_captured_in_a_cuda_graph(dl):
+    """worker_step, aggregate_apply and step_fused neither synchronise nor allocate, so a
+    multi-step loop can be captured once and replayed; the replay must equal the eager steps."""
+    w = inputs.custom([3 * 4096 + 5, 77], 4, MAJ, "f32", lr=1e-2, weight_decay=0.5)
+    dev = torch.device("cuda:0")
+    N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
+    ctx = gp.make_ctx(dl, w)
+    g = inputs.fill_grads(w, 0, torch.empty(N, D)).to(dev)
+    x0 = inputs.fill_x0(w, torch.empty(D)).to(dev)
+
+    def run(eager: bool, fused: bool):
+        m = torch.zeros(N, D, device=dev)
+        x = x0.clone()
+        packed = torch.zeros(N, W, dtype=torch.int32, device=dev)
+
+        def steps():
+            for _ in range(3):
+                if fused:
+                    ctx.step_fused(g, m, x, packed)
+                else:
+                    ctx.worker_step(-1, g, m, packed)
+                    ctx.aggregate_apply(packed, x)
+        if eager:
+            steps()
+        else:
+            side = torch.cuda.Stream()
+            gph = torch.cuda.CUDAGraph()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.graph(gph, stream=side):
+                steps()
+            gph.replay()
+        torch.cuda.synchronize()
+        return m, x, packed
+
+    for fused in (False, True):
+        a, b = run(True, fused), run(False, fused)
+        assert all(torch.equal(u, v) for u, v in zip(a, b))
+    ctx.destroy()
