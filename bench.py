@@ -272,12 +272,21 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    wire = torch.zeros(ctx.delta_planes() * W, dtype=torch.int32, device=dev) if args.path == "wire" else None
+
+    def server_side():
+        if args.path == "wire":                       # vote into the broadcast message, then apply from it
+            ctx.aggregate(packed, wire)
+            ctx.apply_delta(wire, x)
+        else:
+            ctx.aggregate_apply(packed, x)
+
     def step():
         if args.path == "fused":
             ctx.step_fused(g, m, x, None)
         else:
             ctx.worker_step(-1, g, m, packed)
-            ctx.aggregate_apply(packed, x)
+            server_side()
 
     for t in range(args.warmup):
         inputs.fill_grads(w, t, g)
@@ -315,7 +324,7 @@ def run_ours(args):
         else:
             ctx.worker_step(-1, g, m, packed)
             ev[t][1].record(stream)
-            ctx.aggregate_apply(packed, x)
+            server_side()
         ev[t][2].record(stream)
     barrier()
     sampler.window_end()
@@ -384,7 +393,9 @@ def run_ours(args):
         stages = None
         if args.path != "fused":
             b2 = w.d * bytes_per_param_k2(w)
-            stages = {"aggregate_apply_kernel": {"achieved": b2 / (k2 * 1e-3) / 1e9, "unit": "GB/s",
+            if args.path == "wire":                   # votes in, K planes out; K planes in, x in and out
+                b2 += 2 * w.d * ctx.delta_planes() / 8
+            stages = {("aggregate_kernel+apply_delta_kernel" if args.path == "wire" else "aggregate_apply_kernel"): {"achieved": b2 / (k2 * 1e-3) / 1e9, "unit": "GB/s",
                                                  "frac": b2 / (k2 * 1e-3) / 1e9 / peak, "ms_per_launch": k2,
                                                  "algorithmic_bytes_per_launch": b2}}
         cpu = None
@@ -456,7 +467,8 @@ def main():
     ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--n-workers", type=int, default=0, help="override N (the c4 sweep)")
     ap.add_argument("--mode", default=None, choices=["majority", "average"])
-    ap.add_argument("--path", default="two_stage", choices=["two_stage", "fused"])
+    ap.add_argument("--path", default="two_stage", choices=["two_stage", "fused", "wire"],
+                    help="wire: server side as two launches with the broadcast message in between")
     ap.add_argument("--state", default="f32", choices=["f32", "bf16"], help="momentum storage")
     ap.add_argument("--graph", action="store_true", help="also time the K steps replayed from one CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
