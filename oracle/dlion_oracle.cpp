@@ -14,7 +14,9 @@
 //                     last equation of Section 3.2;
 //   * wire format  -- Section 3.2 "Communication Cost" and Table 1: delta_i is a
 //                     binary vector of d bits; Delta is binary (Majority Vote) or
-//                     an integer in {0..N} (Averaging).
+//                     an integer in {0..N} (Averaging);
+//   * Global Lion  -- the full-precision comparison scheme of the appendix
+//                     ("Global Lion Convergence") and Section 5.1.
 //
 // The method is exact arithmetic on given inputs, so the oracle is the
 // definition written out coordinate by coordinate.  The paper does not fix the
@@ -321,6 +323,65 @@ int dlion_oracle_apply_delta(const dlion_oracle_segment* segs, uint32_t nseg, ui
             const float u2 = Delta + u1;
             const float u3 = lr * u2;
             x[j] = xo - u3;
+        }
+    }
+    return 0;
+}
+
+// Global Lion, the full-precision scheme the paper compares against (Appendix,
+// "Global Lion Convergence", the scheme labelled Global Lion; Section 5.1 "G-Lion";
+// Table 1 row "Global Lion/AdamW": 32 d bits each way).  Per coordinate:
+//     mt_i  = beta1 m_i + (1-beta1) g_i                    (old m_i)
+//     m_i  <- beta2 m_i + (1-beta2) g_i
+//     G     = (1/N) sum_i mt_i
+//     x    <- x - eps ( sign(G) + lambda x )
+// Readings: R1 (binary32, one rounding per operation, no FMA) with the sum taken
+// in worker order i = 0, 1, ..., N-1 starting from mt_0, then ONE division by
+// (float)N; R2 for the sign (G >= 0 gives +1); every worker keeps its own m_i as
+// the appendix scheme writes it (Section 5.1's "Lion on the averaged gradients" is
+// the same sequence in exact arithmetic when all m_i start equal).
+//   delta_bits [d_pad/32]  optional: bit = 1 iff sign(G) = +1, padding bits 0
+// Returns 0, or -1 on a malformed argument.
+int dlion_oracle_global_step(const dlion_oracle_segment* segs, uint32_t nseg, uint64_t d_pad,
+                             uint32_t n_workers, int gdtype, const void* g, float* m, float* x,
+                             uint32_t* delta_bits, float beta1, float beta2, float lr,
+                             float weight_decay) {
+    if (!segs || !g || !m || !x || d_pad % 32 != 0 || n_workers == 0) return -1;
+    const float w1 = 1.0f - beta1;                               // R1: (1-beta) in binary32
+    const float w2 = 1.0f - beta2;
+    const float Nf = static_cast<float>(n_workers);
+    for (uint32_t s = 0; s < nseg; ++s) {
+        const uint64_t lo = segs[s].elem_offset;
+        const uint64_t hi = lo + segs[s].numel;
+        if (hi > d_pad || lo % 32 != 0) return -1;
+        for (uint64_t w = lo / 32; w < (hi + 31) / 32; ++w) {
+            uint32_t dword = 0;
+            for (uint32_t b = 0; b < 32; ++b) {
+                const uint64_t j = w * 32 + b;
+                if (j < lo || j >= hi) continue;
+                float total = 0.0f;
+                for (uint32_t i = 0; i < n_workers; ++i) {
+                    const size_t idx = static_cast<size_t>(i) * d_pad + j;
+                    const float gf = load_grad(g, gdtype, idx);
+                    const float mo = m[idx];
+                    const float p1 = beta1 * mo;
+                    const float q1 = w1 * gf;
+                    const float mt = p1 + q1;                    // the blend each worker would send
+                    total = (i == 0) ? mt : total + mt;          // fp32 sum in worker order
+                    const float p2 = beta2 * mo;
+                    const float q2 = w2 * gf;
+                    m[idx] = p2 + q2;
+                }
+                const float G = total / Nf;
+                const float Delta = (G >= 0.0f) ? 1.0f : -1.0f;
+                if (G >= 0.0f) dword |= 1u << b;
+                const float xo = x[j];
+                const float v1 = weight_decay * xo;
+                const float v2 = Delta + v1;
+                const float v3 = lr * v2;
+                x[j] = xo - v3;
+            }
+            if (delta_bits) delta_bits[w] = dword;
         }
     }
     return 0;

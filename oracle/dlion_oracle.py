@@ -73,6 +73,11 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.dlion_oracle_apply_delta.argtypes = [
         ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int,
         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_float]
+    lib.dlion_oracle_global_step.restype = ctypes.c_int
+    lib.dlion_oracle_global_step.argtypes = [
+        ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int,
+        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+        ctypes.c_float, ctypes.c_float, ctypes.c_float, ctypes.c_float]
     return lib
 
 
@@ -199,6 +204,24 @@ def apply_delta(segments, d_pad: int, n_workers: int, mode: int, delta_wire: np.
                                                   _ptr(delta_wire), _ptr(x), lr, weight_decay)
     if rc != 0:
         raise ValueError("dlion_oracle_apply_delta rejected its arguments")
+
+
+def global_step(segments, d_pad: int, n_workers: int, g: np.ndarray, m: np.ndarray, x: np.ndarray,
+                beta1: float, beta2: float, lr: float, weight_decay: float,
+                delta_bits: Optional[np.ndarray] = None, lib: Optional[ctypes.CDLL] = None) -> None:
+    """One step of Global Lion (appendix scheme): fp32 mean of the workers' blends, one sign,
+    the x update; every worker's momentum updated in place."""
+    gdt = {np.dtype(np.float32): GRAD_F32, np.dtype(np.uint16): GRAD_BF16}[g.dtype]
+    _check(g, g.dtype, n_workers * d_pad, "g")
+    _check(m, np.float32, n_workers * d_pad, "m")
+    _check(x, np.float32, d_pad, "x")
+    if delta_bits is not None:
+        _check(delta_bits, np.uint32, d_pad // 32, "delta_bits")
+    rc = (lib or _get()).dlion_oracle_global_step(_segs(segments), len(segments), d_pad, n_workers, gdt,
+                                                  _ptr(g), _ptr(m), _ptr(x), _ptr(delta_bits),
+                                                  beta1, beta2, lr, weight_decay)
+    if rc != 0:
+        raise ValueError("dlion_oracle_global_step rejected its arguments")
 
 
 def has_openmp() -> bool:

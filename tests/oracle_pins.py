@@ -446,8 +446,108 @@ def check_bf16_momentum_store(lib):
     assert np.isnan(widen(nan_state)).all()
 
 
+# ---------------------------------------------------------------- Global Lion (comparison scheme)
+def _hand_rows(name):
+    hp, rows = {}, []
+    for line in open(os.path.join(GOLDEN, name)):
+        line = line.split("#")[0].split()
+        if not line:
+            continue
+        if len(line) == 2:
+            hp[line[0]] = float(line[1])
+        else:
+            rows.append([float(v) for v in line])
+    return hp, rows
+
+
+def check_global_lion_hand_case(lib):
+    """The hand-derived example where the sign of the mean and the majority of the signs differ."""
+    hp, rows = _hand_rows("global_lion_hand_case.txt")
+    segs, d_pad = _flat(1)
+    m = np.zeros((3, d_pad), np.float32)
+    x = np.zeros(d_pad, np.float32)
+    x[0] = hp["x0"]
+    for r in rows:
+        g = np.zeros((3, d_pad), np.float32)
+        g[:, 0] = r[1:4]
+        # the same blends through Distributed Lion's vote (from the same momentum), for the contrast
+        m_d, x_d = m.copy(), x.copy()
+        packed = np.zeros((3, d_pad // 32), np.uint32)
+        dbits_d = np.zeros(d_pad // 32, np.uint32)
+        orc.worker_step(segs, d_pad, 3, g, m_d, packed, hp["beta1"], hp["beta2"], lib=lib)
+        orc.aggregate_apply(segs, d_pad, 3, MAJ, packed, x_d, hp["eps"], hp["lambda"], delta_bits=dbits_d, lib=lib)
+        dbits = np.zeros(d_pad // 32, np.uint32)
+        orc.global_step(segs, d_pad, 3, g, m, x, hp["beta1"], hp["beta2"], hp["eps"], hp["lambda"],
+                        delta_bits=dbits, lib=lib)
+        assert (1 if dbits[0] & 1 else -1) == int(r[4])
+        assert x[0] == np.float32(r[5])
+        assert tuple(m[:, 0]) == tuple(np.float32(v) for v in r[6:9])
+        assert np.array_equal(m, m_d)                              # same momentum rule
+        assert (1 if dbits_d[0] & 1 else -1) == int(r[9]) == -int(r[4])   # the two schemes disagree here
+        assert dbits[0] >> 1 == 0 and not x[1:].any()              # padding untouched
+
+
+def check_global_lion_definition(lib):
+    """Sign of the float64 mean of the float64 blends wherever that mean is clearly non-zero;
+    x from the float64 update within an ulp per operation; momentum equal to the worker step's;
+    N = 1 is Lion (Eq. 1) = Distributed Lion under either rule; N identical workers = one worker."""
+    rng = np.random.default_rng(11)
+    b1, b2, lr, wd = 0.9, 0.99, 1e-2, 0.3
+    for N, d in ((1, 700), (2, 515), (3, 700), (8, 333), (33, 129)):
+        segs, d_pad = _flat(d)
+        m = f32(rng.standard_normal((N, d_pad)) * 0.1)
+        x = f32(rng.standard_normal(d_pad))
+        for t in range(3):
+            g = f32(rng.standard_normal((N, d_pad)))
+            m_old, x_old = m.copy(), x.copy()
+            dbits = np.zeros(d_pad // 32, np.uint32)
+            orc.global_step(segs, d_pad, N, g, m, x, b1, b2, lr, wd, delta_bits=dbits, lib=lib)
+            mt = np.float64(np.float32(b1)) * m_old.astype(np.float64) + (1.0 - np.float64(np.float32(b1))) * g
+            mean = mt.mean(axis=0)
+            clear = np.abs(mean[:d]) > 1e-5
+            assert clear.mean() > 0.9
+            got = unpack(dbits[None, :], d_pad)[0, :d].astype(bool)
+            assert np.array_equal(got[clear], (mean[:d] > 0)[clear])
+            delta = np.where(got, 1.0, -1.0)
+            x64 = x_old[:d].astype(np.float64) - np.float64(np.float32(lr)) * (
+                delta + np.float64(np.float32(wd)) * x_old[:d].astype(np.float64))
+            assert np.abs(x[:d] - x64).max() <= 4 * np.spacing(np.float32(np.abs(x64).max() + 1))
+            m_w = m_old.copy()
+            orc.worker_step(segs, d_pad, N, g, m_w, np.zeros((N, d_pad // 32), np.uint32), b1, b2, lib=lib)
+            assert np.array_equal(m, m_w)
+            assert np.array_equal(x[d:], x_old[d:]) and np.array_equal(m[:, d:], m_old[:, d:])
+            if N == 1:                                             # Lion, Eq. (1)
+                for mode in (MAJ, AVG):
+                    m1, x1 = m_old.copy(), x_old.copy()
+                    pk = np.zeros((1, d_pad // 32), np.uint32)
+                    orc.worker_step(segs, d_pad, 1, g, m1, pk, b1, b2, lib=lib)
+                    orc.aggregate_apply(segs, d_pad, 1, mode, pk, x1, lr, wd, lib=lib)
+                    assert np.array_equal(x, x1) and np.array_equal(dbits, pk[0])
+    # N identical workers reproduce one worker (the sum of N equal values has that value's sign)
+    segs, d_pad = _flat(300)
+    for N in (2, 5, 16):
+        g1 = f32(rng.standard_normal((1, d_pad)))
+        g1[0, :7] = 0.0                                            # exact zeros: sign(0) = +1 either way
+        m1 = f32(rng.standard_normal((1, d_pad)) * 0.1)
+        m1[0, :7] = 0.0
+        x1 = f32(rng.standard_normal(d_pad))
+        mN, xN = np.repeat(m1, N, axis=0), x1.copy()
+        orc.global_step(segs, d_pad, 1, g1, m1, x1, b1, b2, lr, wd, lib=lib)
+        orc.global_step(segs, d_pad, N, np.repeat(g1, N, axis=0), mN, xN, b1, b2, lr, wd, lib=lib)
+        assert np.array_equal(xN, x1) and all(np.array_equal(mN[i], m1[0]) for i in range(N))
+    # bf16 gradients are widened exactly
+    gb = (f32(rng.standard_normal((3, d_pad))).view(np.uint32) >> 16).astype(np.uint16)
+    gf = (gb.astype(np.uint32) << 16).view(np.float32)
+    ma, xa = np.zeros((3, d_pad), np.float32), np.ones(d_pad, np.float32)
+    mb, xb = ma.copy(), xa.copy()
+    orc.global_step(segs, d_pad, 3, gb, ma, xa, b1, b2, lr, wd, lib=lib)
+    orc.global_step(segs, d_pad, 3, gf, mb, xb, b1, b2, lr, wd, lib=lib)
+    assert np.array_equal(xa, xb) and np.array_equal(ma, mb)
+
+
 ALL_CHECKS = [check_hand_case, check_sign_of_zero_and_tie, check_delta_is_sign_of_blend,
               check_single_worker_is_lion, check_identical_workers, check_beta_zero_is_signsgd,
               check_equal_betas_is_signum, check_counts_bruteforce, check_x_closed_form,
               check_phase_one_contraction, check_padding_untouched, check_wire_bits,
-              check_delta_wire_roundtrip, check_per_worker_betas, check_bf16_momentum_store]
+              check_delta_wire_roundtrip, check_per_worker_betas, check_bf16_momentum_store,
+              check_global_lion_hand_case, check_global_lion_definition]

@@ -43,6 +43,21 @@ MUTANTS = {
     "bf16_store_rounds_half_up": ("u += 0x7FFFu + lsb;", "u += 0x8000u;"),
     "betas_of_worker_zero": ("const float beta1 = beta1s[i], beta2 = beta2s[i];",
                              "const float beta1 = beta1s[0], beta2 = beta2s[0];"),
+    "global_blend_uses_beta2": ("const float p1 = beta1 * mo;", "const float p1 = beta2 * mo;"),
+    "global_blend_uses_new_momentum": ("const float p1 = beta1 * mo;", "const float p1 = beta1 * (beta2 * mo + w2 * gf);"),
+    "global_votes_instead_of_mean": ("total = (i == 0) ? mt : total + mt;",
+                                     "total = (i == 0 ? 0.0f : total) + ((mt >= 0.0f) ? 1.0f : -1.0f);"),
+    "global_only_first_worker": ("total = (i == 0) ? mt : total + mt;", "total = (i == 0) ? mt : total;"),
+    "global_one_minus_beta_dropped": ("const float w1 = 1.0f - beta1;                               // R1: (1-beta) in binary32",
+                                      "const float w1 = 1.0f;"),
+    "global_sign_negated": ("const float Delta = (G >= 0.0f) ? 1.0f : -1.0f;",
+                            "const float Delta = (G >= 0.0f) ? -1.0f : 1.0f;"),
+    "global_momentum_not_updated": ("m[idx] = p2 + q2;", "m[idx] = mo;"),
+    "global_momentum_uses_beta1": ("m[idx] = p2 + q2;", "m[idx] = p1 + q1;"),
+    "global_weight_decay_sign": ("const float v2 = Delta + v1;", "const float v2 = Delta - v1;"),
+    "global_update_sign": ("x[j] = xo - v3;", "x[j] = xo + v3;"),
+    "global_sums_gradients_only": ("const float mt = p1 + q1;                    // the blend each worker would send",
+                                   "const float mt = gf;"),
     "average_down_bits_floor_log": ("while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;",
                                     "while ((2ull << bits) <= static_cast<uint64_t>(n_workers)) ++bits;"),
 }
