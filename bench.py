@@ -428,6 +428,82 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def make_packed(ctx, dlion, w, dev, step: int = 0, rounds: int = 1):
+    """The wire buffer [N][d_pad/32] of workload w without holding N gradient and
+    momentum arenas: the workers are stepped one at a time through
+    dlion_worker_step(i) on one worker-sized gradient buffer (each worker's own
+    seeded gradients; `rounds` steps from m = 0)."""
+    N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
+    gdt = inputs.grad_torch_dtype(w)
+    packed = torch.zeros(N, W, dtype=torch.int32, device=dev)
+    g1 = torch.empty(1, D, dtype=gdt, device=dev)
+    m1 = torch.empty(D, dtype=torch.float32, device=dev)
+    for i in range(N):
+        m1.zero_()
+        for t in range(rounds):
+            inputs.fill_grads(w, step + t, g1, workers=[i])
+            ctx.worker_step(i, g1[0], m1, packed[i])
+    torch.cuda.synchronize()
+    return packed
+
+
+def run_server_stage(args):
+    """Times the server-side kernel alone (dlion_aggregate_apply) on the wire buffer of
+    the workload: N*d/8 B of votes plus x are all the device memory it needs, so even
+    the large-N cases are small enough to profile."""
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    from paper_2404_00438_b200 import build
+    build.build()
+    from paper_2404_00438_b200 import dlion
+    w = inputs.workload(args.workload)
+    if args.n_workers:
+        w.n_workers = args.n_workers
+    mode = mode_of(args.mode) if args.mode else w.mode
+    N, D = w.n_workers, w.d_pad
+    ctx = dlion.Dlion(w.segments, D, N, w.beta1, w.beta2, w.lr, w.weight_decay, mode,
+                      dlion.GRAD_F32 if w.grad_dtype == "f32" else dlion.GRAD_BF16)
+    packed = make_packed(ctx, dlion, w, dev)
+    x = inputs.fill_x0(w, torch.empty(D, device=dev))
+    stream = torch.cuda.current_stream()
+    for _ in range(max(args.warmup, 3)):
+        ctx.aggregate_apply(packed, x)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    sampler.window_start()
+    ev[0].record(stream)
+    for t in range(args.steps):
+        ctx.aggregate_apply(packed, x)
+        ev[t + 1].record(stream)
+    torch.cuda.synchronize()
+    sampler.window_end()
+    clocks = sampler.stop()
+    ms = [ev[t].elapsed_time(ev[t + 1]) for t in range(args.steps)]
+    k2 = statistics.mean(ms)
+    peak, peak_src = measured_peak()
+    b2 = w.d * bytes_per_param_k2(w)
+    achieved = b2 / (k2 * 1e-3) / 1e9
+    line = {
+        "metric": "dlion_server_stage_params_per_s", "value": w.d / (k2 * 1e-3) / 1e9, "unit": "G param/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": k2,
+        "ms_min": min(ms), "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "n_workers": N, "d": w.d, "stage": "server",
+                   "mode": "average" if mode else "majority",
+                   "l2": "votes + x = %.0f MB, larger than L2" % ((N * D / 8 + 4 * D) / 1e6)},
+        "roofline": {"bound": "hbm", "kernel": "aggregate_apply_kernel", "achieved": achieved, "peak": 8000.0,
+                     "unit": "GB/s", "frac": achieved / 8000.0, "peak_source": "nominal 8 TB/s",
+                     "vs_measured_copy": achieved / peak, "measured_copy_gbs": peak, "measured_copy_source": peak_src,
+                     "algorithmic_bytes_per_launch": b2, "ms_per_launch": k2, "traffic": None},
+        "gpu_launches": args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    ctx.destroy()
+
+
 def run_e2e(args, ctx, w, mode, g, m, x, packed, dev, world, barrier):
     """dlion_step_host: per step, N*D gradient elements host->device, Delta device->host."""
     import torch.distributed as dist
@@ -435,7 +511,7 @@ def run_e2e(args, ctx, w, mode, g, m, x, packed, dev, world, barrier):
     host_g = torch.empty(N, D, dtype=g.dtype, pin_memory=True)
     host_g.copy_(g)
     staging = torch.empty(2, D, dtype=g.dtype, device=dev)
-    wire_bytes = D if mode == inputs.AVERAGE else W * 4
+    wire_bytes = ctx.delta_planes() * W * 4           # the broadcast message: 1 or K planes of d bits
     wire = torch.zeros(wire_bytes, dtype=torch.uint8, device=dev)
     host_wire = torch.zeros(wire_bytes, dtype=torch.uint8, pin_memory=True)
     stream = torch.cuda.current_stream()
@@ -470,6 +546,8 @@ def main():
     ap.add_argument("--path", default="two_stage", choices=["two_stage", "fused", "wire"],
                     help="wire: server side as two launches with the broadcast message in between")
     ap.add_argument("--state", default="f32", choices=["f32", "bf16"], help="momentum storage")
+    ap.add_argument("--stage", default="step", choices=["step", "server"],
+                    help="server: time the server-side kernel alone on the workload's wire buffer (1 GPU)")
     ap.add_argument("--graph", action="store_true", help="also time the K steps replayed from one CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -481,6 +559,8 @@ def main():
         args.warmup = 3                               # timing hygiene: at least three warm-up steps
     if args.impl == "reference":
         run_reference(args)
+    elif args.stage == "server":
+        run_server_stage(args)
     else:
         run_ours(args)
 

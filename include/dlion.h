@@ -54,7 +54,7 @@ extern "C" {
 
 #define DLION_ALIGN 128u        /* elements: alignment of segment starts and of d_pad */
 #define DLION_MAX_WORKERS 65535u /* up to 16 bit planes of votes */
-#define DLION_MAX_WORKERS_BYTE_COUNTS 255u /* count_out, dlion_step_fused, dlion_step_static, dlion_step_host with Averaging */
+#define DLION_MAX_WORKERS_BYTE_COUNTS 255u /* count_out of dlion_aggregate_apply (one byte per count) */
 #define DLION_STATIC_MAX_COORD_WORKERS 134217728ull /* dlion_step_static: limit on N * d_pad */
 
 typedef struct dlion_ctx dlion_ctx; /* opaque; host-side object */
@@ -169,6 +169,22 @@ uint32_t dlion_delta_planes(const dlion_ctx* ctx);
 dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float* x,
                               uint32_t* packed_out, void* cuda_stream);
 
+/* Global Lion, the full-precision scheme the paper compares Distributed Lion with
+ * (appendix "Global Lion Convergence", the scheme labelled Global Lion; Section 5.1
+ * "G-Lion"; Table 1 row "Global Lion/AdamW", 32 d bits each way), in one launch:
+ *     mt_i = beta1 m_i + (1-beta1) g_i  (old m_i);   m_i <- beta2 m_i + (1-beta2) g_i
+ *     x   <- x - eps ( sign( (1/N) sum_i mt_i ) + lambda x )
+ * Arithmetic as in the conventions above: the sum is taken in binary32 in worker
+ * order starting from mt_0, divided once by (float)N, and sign(v) = +1 for v >= 0.
+ * It is here as the measured denominator of the comparison (time per step, and
+ * dlion_wire_bytes(ctx, 2) for what it would send); the mode of the context is
+ * not used.  fp32 momentum and one (beta1, beta2) for all workers only:
+ * DLION_EINVAL after dlion_set_momentum_dtype(bf16) or dlion_set_worker_betas.
+ *   grads [N][d_pad] in; m [N][d_pad] in/out; x [d_pad] in/out
+ *   delta_bits_out  out, nullable  [d_pad/32]: bit = 1 iff the sign is +1 */
+dlion_status dlion_step_global(dlion_ctx* ctx, const void* grads, float* m, float* x,
+                               uint32_t* delta_bits_out, void* cuda_stream);
+
 /* One whole step with the gradients in HOST memory (pinned memory makes the
  * copies asynchronous).  Worker i's gradients are copied to the device while
  * worker i-1's are being consumed by the worker-side kernel; after the last
@@ -176,10 +192,14 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float*
  *   host_grads      in, host   [N][d_pad] gradients
  *   m, x, packed    device     as above (packed is used as the wire buffer)
  *   staging         device     2 * d_pad gradient elements (two slices)
- *   delta_wire_dev  device, nullable  [d_pad/32] words (Majority Vote) or
- *                   [d_pad] bytes (Averaging, N <= 255): Delta as the server sends it
- *   host_delta_out  out, host, nullable: copy of delta_wire_dev; needs
- *                   delta_wire_dev.  Complete when cuda_stream's work is.
+ *   delta_wire_dev  device, nullable  the broadcast message in the format of
+ *                   dlion_aggregate: dlion_delta_planes(ctx) planes of d_pad/32 words
+ *                   (one plane of Delta bits for Majority Vote, the K count planes
+ *                   for Averaging; any N)
+ *   host_delta_out  out, host, nullable: copy of delta_wire_dev (planes * d_pad/8
+ *                   bytes); needs delta_wire_dev.  Complete when cuda_stream's work is.
+ * Every argument is checked before anything is enqueued: a rejected call leaves
+ * m, packed and x untouched.
  * Uses one internal copy stream ordered against cuda_stream by events. */
 dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, void* m, float* x,
                              uint32_t* packed, void* staging, void* delta_wire_dev,
@@ -192,21 +212,25 @@ dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, void* m, fl
  * call cudaMalloc where they step the optimizer: a host whose allocator already
  * owns all device memory, a latency-critical loop that cannot take cudaMalloc's
  * device-wide synchronisation, or a plug-in restricted to the buffers it is
- * handed.  The segment table and the 1-bit wire buffer live in a fixed array
- * inside the library image (16 MiB + 256 B per GPU that loads the library, held
- * until the process exits).  The call allocates nothing, on host or device.
- *   d, n_workers   the problem (n_workers <= 255); d_pad = d rounded up to DLION_ALIGN, and
+ * handed.  The 1-bit wire buffer is a fixed 16 MiB array inside the library image
+ * (held, until the process exits, by every GPU on which the library's device
+ * code has been loaded), and a flat vector needs no tile table.
+ * The FIRST call on a device is a set-up call: the CUDA runtime loads the
+ * library's device code then (which is when the array is reserved, and can fail
+ * with DLION_ECUDA if the device is already full) and the array's device address
+ * is looked up, with that device current.  Make it at start-up, before another
+ * allocator takes the remaining memory and before any stream capture begins.
+ * Every later call allocates nothing, on host or device.
+ *   d, n_workers   the problem; d_pad = d rounded up to DLION_ALIGN, and
  *                  n_workers * d_pad <= DLION_STATIC_MAX_COORD_WORKERS, else
  *                  DLION_EINVAL ("does not fit the fixed scratch")
  *   grads [N][d_pad], m [N][d_pad] (in/out), x [d_pad] (in/out): device, 16-byte
  *                  aligned, as for dlion_worker_step(-1) / dlion_aggregate_apply
  * Results are those of dlion_worker_step(-1) + dlion_aggregate_apply with the
- * same hyper-parameters.  The first call on each device looks up the array's
- * device address (that device must be current); make that first call before
- * any stream capture begins.  All calls on a device share the array and it keeps
- * the last call's bits: every word the step reads is rewritten first, so nothing
- * needs clearing, but two calls that overlap on the GPU (different streams, no
- * ordering) race on it and give undefined results. */
+ * same hyper-parameters (fp32 momentum, one beta pair).  All calls on a device
+ * share the array and it keeps the last call's bits: every word the step reads is
+ * rewritten first, so nothing needs clearing, but two calls that overlap on the
+ * GPU (different streams, no ordering) race on it and give undefined results. */
 dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float beta1, float beta2,
                                float lr, float weight_decay, dlion_mode mode,
                                dlion_gdtype gdtype, const void* grads, float* m, float* x,

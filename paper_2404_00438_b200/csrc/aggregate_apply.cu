@@ -13,8 +13,12 @@
 // even at N = 128.  Majority Vote then needs one bitwise comparison of the planes
 // with ceil(N/2), which yields the Delta word directly.  For the update the warp
 // walks its 1024 coordinates in eight 128-coordinate chunks (lane l: coordinates
-// 4l..4l+3, one 16-byte access) and fetches the needed plane bits from the owning
-// lane with a shuffle.
+// 4l..4l+3, one 16-byte access).  Majority Vote fetches its four Delta bits from
+// the owning lane with one shuffle per chunk.  Averaging needs the counts
+// themselves: the owning lane transposes its planes into one byte per coordinate
+// (word-wide delta swaps) and hands them over through shared memory, so a
+// consumer pays one 16-byte shared load per chunk and one byte permute plus one
+// table lookup per coordinate.
 //
 // HBM traffic per coordinate: N/8 B of votes + 4 B read + 4 B write of x
 // (+ 1/8 B Delta bits, + 1 B count when requested).
@@ -24,11 +28,17 @@ namespace dlion {
 namespace {
 
 constexpr int kThreads = 128;             // 4 warps x 1024 coordinates = one tile
+constexpr int kWarps = kThreads / 32;
 constexpr int kMinBlocks = 6;             // register budget: 6 blocks (24 warps) per SM; 4 once N >= 64
+
+__device__ __forceinline__ uint32_t pack_counts(const Counts4& k) {          // N <= 255: one byte each
+    return k.c[0] | (k.c[1] << 8) | (k.c[2] << 16) | (k.c[3] << 24);
+}
+
 // Last tile of a segment: every access guarded against the segment's end.
 template <int PLANES, bool AVG, bool COUNTS>
 __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, uint32_t warp, uint32_t lane,
-                                         uint32_t thr, const float* avg_table) {
+                                         uint32_t thr, const float* avg_table, CountArea<(PLANES > 8)>* area) {
     const uint32_t w0 = warp * kWarpSpan;
     if (w0 >= t.valid) return;                                  // warp-uniform
     const uint32_t my0 = w0 + lane * 32;                        // first coordinate of my word
@@ -39,14 +49,23 @@ __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, ui
     count_votes<PLANES>(pl, p.packed + word_idx, p.w_stride, p.n_workers, nbits != 0);
     const uint32_t dword = planes_ge<PLANES>(pl, thr) & vmask;
     if (p.delta_bits != nullptr && nbits != 0) p.delta_bits[word_idx] = dword;
+    if constexpr (COUNTS) publish_counts<PLANES>(pl, area, lane);
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
-        const Votes4 v = my_votes<PLANES, COUNTS>(pl, dword, c, lane);
+        Counts4 k;
+        uint32_t dn = 0;
+        if constexpr (COUNTS) k = my_counts<PLANES>(area, c, lane);
+        else dn = my_delta_bits(dword, c, lane);
         const uint32_t j0 = w0 + c * kChunk + lane * 4;
         const unsigned long long e = t.base + j0;
         for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
-            p.x[e + q] = apply_coord(p.x[e + q], delta_value<PLANES, AVG>(v, q, avg_table, p.n_workers), p.lr, p.wd);
-            if (p.count != nullptr) p.count[e + q] = static_cast<uint8_t>(count_of<PLANES>(v, q));
+            float delta;
+            if constexpr (COUNTS) delta = delta_of_count<PLANES, AVG>(k.c[q], thr, avg_table, p.n_workers);
+            else delta = ((dn >> q) & 1u) ? 1.0f : -1.0f;
+            p.x[e + q] = apply_coord(p.x[e + q], delta, p.lr, p.wd);
+            if constexpr (COUNTS) {
+                if (p.count != nullptr) p.count[e + q] = static_cast<uint8_t>(k.c[q]);
+            }
         }
     }
 }
@@ -58,12 +77,14 @@ __global__ void __launch_bounds__(kThreads, PLANES >= 7 ? 4 : kMinBlocks)
 aggregate_apply_kernel(const __grid_constant__ AggParams p) {
     // Delta of Averaging for every count P, one private copy per warp: it is
     // filled after the tile's first loads are in flight and needs no block barrier.
-    __shared__ float avg_tables[(AVG && PLANES <= 8) ? kThreads / 32 : 1][(AVG && PLANES <= 8) ? 256 : 1];
+    __shared__ float avg_tables[(AVG && PLANES <= 8) ? kWarps : 1][(AVG && PLANES <= 8) ? 256 : 1];
+    __shared__ CountArea<(PLANES > 8)> areas[COUNTS ? kWarps : 1];
     const uint32_t n = p.n_workers;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t thr = (n + 1u) >> 1;   // 2P >= N  <=>  P >= ceil(N/2)
     float* avg_table = avg_tables[(AVG && PLANES <= 8) ? warp : 0];
+    CountArea<(PLANES > 8)>* area = &areas[COUNTS ? warp : 0];
     bool have_table = !AVG;
     auto fill_table = [&]() {
         fill_avg_table<PLANES>(avg_table, n, lane);
@@ -71,10 +92,10 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
     };
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.flat_d, tile);
         if (t.valid != kTile) {
             if (!have_table) fill_table();
-            ragged_tile<PLANES, AVG, COUNTS>(p, t, warp, lane, thr, avg_table);
+            ragged_tile<PLANES, AVG, COUNTS>(p, t, warp, lane, thr, avg_table, area);
             continue;
         }
         // ---- full tile: x loads first (they do not depend on the votes), then
@@ -87,20 +108,33 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
         if (!have_table) fill_table();
         uint32_t pl[kMaxPlanes];
         count_votes<PLANES>(pl, p.packed + word_idx, p.w_stride, n, true);
-        const uint32_t dword = planes_ge<PLANES>(pl, thr);
+        uint32_t dword = 0;
+        if (!COUNTS || p.delta_bits != nullptr) dword = planes_ge<PLANES>(pl, thr);
         if (p.delta_bits != nullptr) p.delta_bits[word_idx] = dword;
+        if constexpr (COUNTS) publish_counts<PLANES>(pl, area, lane);
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            const Votes4 vt = my_votes<PLANES, COUNTS>(pl, dword, c, lane);
-            float4 v = xv[c];
-            v.x = apply_coord(v.x, delta_value<PLANES, AVG>(vt, 0, avg_table, n), p.lr, p.wd);
-            v.y = apply_coord(v.y, delta_value<PLANES, AVG>(vt, 1, avg_table, n), p.lr, p.wd);
-            v.z = apply_coord(v.z, delta_value<PLANES, AVG>(vt, 2, avg_table, n), p.lr, p.wd);
-            v.w = apply_coord(v.w, delta_value<PLANES, AVG>(vt, 3, avg_table, n), p.lr, p.wd);
-            *reinterpret_cast<float4*>(p.x + xe + c * kChunk) = v;
+            float d0, d1, d2, d3;
             if constexpr (COUNTS) {
-                if (p.count != nullptr) *reinterpret_cast<uint32_t*>(p.count + xe + c * kChunk) = vt.lo;   // N <= 255 here
+                const Counts4 k = my_counts<PLANES>(area, c, lane);
+                d0 = delta_of_count<PLANES, AVG>(k.c[0], thr, avg_table, n);
+                d1 = delta_of_count<PLANES, AVG>(k.c[1], thr, avg_table, n);
+                d2 = delta_of_count<PLANES, AVG>(k.c[2], thr, avg_table, n);
+                d3 = delta_of_count<PLANES, AVG>(k.c[3], thr, avg_table, n);
+                if (p.count != nullptr) *reinterpret_cast<uint32_t*>(p.count + xe + c * kChunk) = pack_counts(k);   // N <= 255 here
+            } else {
+                const uint32_t dn = my_delta_bits(dword, c, lane);
+                d0 = (dn & 1u) ? 1.0f : -1.0f;
+                d1 = (dn & 2u) ? 1.0f : -1.0f;
+                d2 = (dn & 4u) ? 1.0f : -1.0f;
+                d3 = (dn & 8u) ? 1.0f : -1.0f;
             }
+            float4 v = xv[c];
+            v.x = apply_coord(v.x, d0, p.lr, p.wd);
+            v.y = apply_coord(v.y, d1, p.lr, p.wd);
+            v.z = apply_coord(v.z, d2, p.lr, p.wd);
+            v.w = apply_coord(v.w, d3, p.lr, p.wd);
+            *reinterpret_cast<float4*>(p.x + xe + c * kChunk) = v;
         }
     }
 }
@@ -123,24 +157,7 @@ cudaError_t launch(const AggParams& p, cudaStream_t s) {
 
 cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s) {
     (void)sm_count;
-    switch (planes_for(p.n_workers)) {    // planes = bit length of N
-        case 1: return launch<1>(p, s);
-        case 2: return launch<2>(p, s);
-        case 3: return launch<3>(p, s);
-        case 4: return launch<4>(p, s);
-        case 5: return launch<5>(p, s);
-        case 6: return launch<6>(p, s);
-        case 7: return launch<7>(p, s);
-        case 8: return launch<8>(p, s);
-        case 9: return launch<9>(p, s);
-        case 10: return launch<10>(p, s);
-        case 11: return launch<11>(p, s);
-        case 12: return launch<12>(p, s);
-        case 13: return launch<13>(p, s);
-        case 14: return launch<14>(p, s);
-        case 15: return launch<15>(p, s);
-        default: return launch<16>(p, s);
-    }
+    return dispatch_planes(p.n_workers, [&](auto planes) { return launch<decltype(planes)::value>(p, s); });
 }
 
 }  // namespace dlion

@@ -61,19 +61,14 @@ dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nse
 
     dlion_ctx* c = new (std::nothrow) dlion_ctx;
     if (c == nullptr) return DLION_ENOMEM;
-    std::vector<dlion::SegDev> rows;
     try {
         c->segs.assign(segs, segs + nseg);
-        rows.resize(nseg);
     } catch (...) {
         delete c;
         return DLION_ENOMEM;
     }
     unsigned long long tiles = 0;
     for (uint32_t s = 0; s < nseg; ++s) {
-        rows[s].elem_offset = segs[s].elem_offset;
-        rows[s].numel = segs[s].numel;
-        rows[s].first_tile = tiles;
         tiles += (segs[s].numel + dlion::kTile - 1) / dlion::kTile;
         c->d += segs[s].numel;
     }
@@ -94,23 +89,11 @@ dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nse
         delete c;
         return DLION_ECUDA;
     }
-    e = cudaMalloc(reinterpret_cast<void**>(&c->segs_dev), sizeof(dlion::SegDev) * nseg);
-    if (e != cudaSuccess) {
-        delete c;
-        return e == cudaErrorMemoryAllocation ? DLION_ENOMEM : DLION_ECUDA;
-    }
-    e = cudaMemcpy(c->segs_dev, rows.data(), sizeof(dlion::SegDev) * nseg, cudaMemcpyHostToDevice);
-    if (e != cudaSuccess) {
-        cudaFree(c->segs_dev);
-        delete c;
-        return DLION_ECUDA;
-    }
     if (tiles != 0) {
         std::vector<dlion::TileRow> trows;
         try {
             trows.reserve(tiles);
         } catch (...) {
-            cudaFree(c->segs_dev);
             delete c;
             return DLION_ENOMEM;
         }
@@ -119,7 +102,7 @@ dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nse
                 dlion::TileRow r;
                 r.base = segs[s].elem_offset + off;
                 r.valid = static_cast<uint32_t>(segs[s].numel - off < dlion::kTile ? segs[s].numel - off : dlion::kTile);
-                r.reserved = 0;
+                r.tensor = s;
                 trows.push_back(r);
             }
         }
@@ -129,7 +112,6 @@ dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nse
         }
         if (e != cudaSuccess) {
             if (c->tiles_dev != nullptr) cudaFree(c->tiles_dev);
-            cudaFree(c->segs_dev);
             delete c;
             return e == cudaErrorMemoryAllocation ? DLION_ENOMEM : DLION_ECUDA;
         }
@@ -193,9 +175,8 @@ dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, vo
     p.g = grads;
     p.m = m;
     p.packed = packed;
-    p.segs = ctx->segs_dev;
     p.tiles = ctx->tiles_dev;
-    p.nseg = ctx->nseg;
+    p.flat_d = 0;
     p.n_workers = worker < 0 ? ctx->n_workers : 1u;
     p.ntiles = ctx->ntiles;
     p.d_pad = ctx->d_pad;
@@ -224,9 +205,8 @@ dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float
     p.x = x;
     p.delta_bits = delta_bits_out;
     p.count = count_out;
-    p.segs = ctx->segs_dev;
     p.tiles = ctx->tiles_dev;
-    p.nseg = ctx->nseg;
+    p.flat_d = 0;
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
     p.w_stride = ctx->d_pad / 32;
@@ -253,9 +233,8 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float*
     p.m = m;
     p.x = x;
     p.packed = packed_out;
-    p.segs = ctx->segs_dev;
     p.tiles = ctx->tiles_dev;
-    p.nseg = ctx->nseg;
+    p.flat_d = 0;
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
     p.d_pad = ctx->d_pad;
@@ -267,6 +246,35 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float*
     p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
     const cudaError_t e = dlion::launch_step_fused(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
                                                    static_cast<cudaStream_t>(cuda_stream));
+    if (e != cudaSuccess) return DLION_ECUDA;
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+dlion_status dlion_step_global(dlion_ctx* ctx, const void* grads, float* m, float* x,
+                               uint32_t* delta_bits_out, void* cuda_stream) {
+    if (ctx == nullptr || grads == nullptr || m == nullptr || x == nullptr) return DLION_EINVAL;
+    if (ctx->sdtype != DLION_STATE_F32 || !ctx->betas.empty()) return DLION_EINVAL;   // one beta pair, fp32 momentum
+    if (!aligned(grads, 16) || !aligned(m, 16) || !aligned(x, 16) || !aligned(delta_bits_out, 16)) {
+        return DLION_EALIGN;
+    }
+    const dlion_status ds = device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    dlion::GlobalParams p;
+    p.g = grads;
+    p.m = m;
+    p.x = x;
+    p.delta_bits = delta_bits_out;
+    p.tiles = ctx->tiles_dev;
+    p.flat_d = 0;
+    p.n_workers = ctx->n_workers;
+    p.ntiles = ctx->ntiles;
+    p.d_pad = ctx->d_pad;
+    p.k = betas_of(ctx);
+    p.lr = ctx->lr;
+    p.wd = ctx->wd;
+    const cudaError_t e = dlion::launch_step_global(p, ctx->gdtype == DLION_GRAD_BF16,
+                                                    static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return DLION_ECUDA;
     if (ctx->ntiles != 0) ctx->launches += 1;
     return DLION_OK;

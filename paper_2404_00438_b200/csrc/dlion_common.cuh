@@ -18,49 +18,46 @@ constexpr uint32_t kTile = 4096;        // coordinates per work item (all kernel
 constexpr uint32_t kChunk = 128;        // coordinates one warp covers per vector access
 constexpr uint32_t kFull = 0xFFFFFFFFu;
 
-// One row per segment, in device memory.  first_tile is the running count of
-// tiles of the segments before it (a tile never spans two segments).
-struct SegDev {
-    unsigned long long elem_offset;
-    unsigned long long numel;
-    unsigned long long first_tile;
-};
-
 struct TileRef {
     unsigned long long base;   // arena index of the tile's first coordinate
     uint32_t valid;            // parameters in the tile, 1..kTile
+    uint32_t tensor;           // index of the segment (tensor) the tile belongs to
 };
 
-// Optional one-row-per-tile table (built by dlion_init): turns the lookup into a
-// single 16-byte load.  Contexts without it (the fixed-scratch step) search.
+// One row per tile (built by dlion_init): a block finds its tile with a single
+// 16-byte load.  A tile never spans two segments.
 struct TileRow {
     unsigned long long base;   // arena index of the tile's first coordinate
     uint32_t valid;            // parameters in the tile, 1..kTile
-    uint32_t reserved;
+    uint32_t tensor;           // segment index
 };
 
-// Largest s with segs[s].first_tile <= tile (segments with numel = 0 own no tile
-// and are never selected because the next row has the same first_tile).
-__device__ __forceinline__ TileRef find_tile(const TileRow* __restrict__ tiles, const SegDev* __restrict__ segs,
-                                             uint32_t nseg, unsigned long long tile) {
+// Tile lookup.  With a table: one load.  Without one the parameters are a flat
+// vector of flat_d coordinates starting at arena index 0 (the fixed-scratch step,
+// which owns no table): plain arithmetic.
+// (Kept out of line on purpose: inlined into the worker-side kernel it changed the
+// register allocation of the whole kernel from 48 to 64 registers, one block less
+// per SM, and the c5 step from 30 to 34 ms.)
+static __device__ __noinline__ TileRef flat_tile(unsigned long long flat_d, unsigned long long tile) {
+    TileRef t;
+    t.base = tile * kTile;
+    const unsigned long long left = flat_d - t.base;
+    t.valid = left < kTile ? static_cast<uint32_t>(left) : kTile;
+    t.tensor = 0;
+    return t;
+}
+
+__device__ __forceinline__ TileRef find_tile(const TileRow* __restrict__ tiles, unsigned long long flat_d,
+                                             unsigned long long tile) {
+    TileRef t;
     if (tiles != nullptr) {
         const uint4 r = __ldg(reinterpret_cast<const uint4*>(tiles + tile));
-        TileRef t;
         t.base = static_cast<unsigned long long>(r.x) | (static_cast<unsigned long long>(r.y) << 32);
         t.valid = r.z;
+        t.tensor = r.w;
         return t;
     }
-    uint32_t lo = 0, hi = nseg;          // answer in [lo, hi)
-    while (hi - lo > 1) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (__ldg(&segs[mid].first_tile) <= tile) lo = mid; else hi = mid;
-    }
-    const unsigned long long off = (tile - __ldg(&segs[lo].first_tile)) * kTile;
-    const unsigned long long left = __ldg(&segs[lo].numel) - off;
-    TileRef t;
-    t.base = __ldg(&segs[lo].elem_offset) + off;
-    t.valid = left < kTile ? static_cast<uint32_t>(left) : kTile;
-    return t;
+    return flat_tile(flat_d, tile);
 }
 
 // Algorithm 1, worker side, one coordinate: returns the sign bit of
@@ -180,9 +177,8 @@ struct WorkerParams {
     const void* g;
     void* m;                         // float, or bf16 when m_bf16
     uint32_t* packed;
-    const SegDev* segs;
-    const TileRow* tiles;            // per-tile rows (device), or null: search segs
-    uint32_t nseg;
+    const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
+    unsigned long long flat_d;
     uint32_t n_workers;              // workers this launch covers (1 for a single-worker call)
     unsigned long long ntiles;       // tiles per worker
     unsigned long long d_pad;        // elements between consecutive workers in g and m
@@ -197,9 +193,8 @@ struct AggParams {
     float* x;
     uint32_t* delta_bits;            // nullable
     uint8_t* count;                  // nullable
-    const SegDev* segs;
-    const TileRow* tiles;            // per-tile rows (device), or null: search segs
-    uint32_t nseg;
+    const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
+    unsigned long long flat_d;
     uint32_t n_workers;
     unsigned long long ntiles;
     unsigned long long w_stride;     // words between consecutive workers in packed
@@ -212,9 +207,8 @@ struct FusedParams {
     void* m;                         // float, or bf16 when m_bf16
     float* x;
     uint32_t* packed;                // nullable
-    const SegDev* segs;
-    const TileRow* tiles;            // per-tile rows (device), or null: search segs
-    uint32_t nseg;
+    const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
+    unsigned long long flat_d;
     uint32_t n_workers;
     unsigned long long ntiles;
     unsigned long long d_pad;
@@ -225,17 +219,32 @@ struct FusedParams {
     int average;
 };
 
+struct GlobalParams {                // Global-Lion comparison step
+    const void* g;
+    float* m;
+    float* x;
+    uint32_t* delta_bits;            // nullable
+    const TileRow* tiles;
+    unsigned long long flat_d;
+    uint32_t n_workers;
+    unsigned long long ntiles;
+    unsigned long long d_pad;
+    Betas k;
+    float lr, wd;
+};
+
 struct WireParams {                  // server-only aggregate / worker-side apply
     const uint32_t* packed;          // aggregate: the N binary vectors
     uint32_t* wire_out;              // aggregate: the broadcast message
     const uint32_t* wire_in;         // apply: the broadcast message
     float* x;                        // apply: parameters
-    const SegDev* segs;
-    const TileRow* tiles;            // per-tile rows (device), or null: search segs
-    uint32_t nseg;
+    const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
+    unsigned long long flat_d;
     uint32_t n_workers;
     unsigned long long ntiles;
-    unsigned long long w_stride;     // words per binary vector / per plane (d_pad / 32)
+    unsigned long long w_stride;     // words between consecutive binary vectors in packed
+    unsigned long long plane_stride; // words between consecutive planes of the message
+    uint32_t kplanes;                // planes in the message: 1, or ceil(log2(N+1)) for Averaging
     float lr, wd;
     int average;
 };
@@ -251,6 +260,7 @@ cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, c
 cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s);
 cudaError_t launch_step_fused(const FusedParams& p, bool bf16, int sm_count, cudaStream_t s);
 cudaError_t launch_wire(const WireParams& p, bool apply, cudaStream_t s);
+cudaError_t launch_step_global(const GlobalParams& p, bool bf16, cudaStream_t s);
 uint32_t planes_for(uint32_t n_workers);   // ceil(log2(N+1))
 
 }  // namespace dlion

@@ -7,7 +7,6 @@
 
 struct dlion_ctx {
     std::vector<dlion_segment> segs;
-    dlion::SegDev* segs_dev = nullptr;
     dlion::TileRow* tiles_dev = nullptr;     // one row per tile
     uint32_t nseg = 0;
     unsigned long long ntiles = 0;

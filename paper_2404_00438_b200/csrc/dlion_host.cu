@@ -6,15 +6,32 @@ namespace {
 
 using dlion::aligned16;
 
-// Streams and events of the copy pipeline; created once, on first use.
+void drop_pipeline(dlion_ctx* c) {
+    for (int k = 0; k < 2; ++k) {
+        if (c->copied[k] != nullptr) cudaEventDestroy(c->copied[k]);
+        if (c->consumed[k] != nullptr) cudaEventDestroy(c->consumed[k]);
+        c->copied[k] = nullptr;
+        c->consumed[k] = nullptr;
+    }
+    if (c->entry != nullptr) cudaEventDestroy(c->entry);
+    c->entry = nullptr;
+    if (c->copy_stream != nullptr) cudaStreamDestroy(c->copy_stream);
+    c->copy_stream = nullptr;
+}
+
+// Streams and events of the copy pipeline; created once, on first use.  All or
+// nothing: a partial failure destroys what was created, so a later call starts
+// over instead of running with missing events.
 cudaError_t ensure_pipeline(dlion_ctx* c) {
     if (c->copy_stream != nullptr) return cudaSuccess;
     cudaError_t e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    if (e != cudaSuccess) c->copy_stream = nullptr;
     for (int k = 0; k < 2 && e == cudaSuccess; ++k) {
         e = cudaEventCreateWithFlags(&c->copied[k], cudaEventDisableTiming);
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->consumed[k], cudaEventDisableTiming);
     }
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->entry, cudaEventDisableTiming);
+    if (e != cudaSuccess) drop_pipeline(c);
     return e;
 }
 
@@ -65,14 +82,22 @@ dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, void* m, fl
         if (st != DLION_OK) return st;
         if (cudaEventRecord(ctx->consumed[b], main) != cudaSuccess) return DLION_ECUDA;
     }
+    // Server side.  The broadcast message, when asked for, is in the format of
+    // dlion_aggregate: one plane of Delta bits (Majority Vote) or the K count planes
+    // (Averaging; vote and update are then two launches with the message in between).
     const bool avg = ctx->mode == DLION_AVERAGE;
-    const dlion_status st = dlion_aggregate_apply(ctx, packed, x,
-                                                  avg ? nullptr : static_cast<uint32_t*>(delta_wire_dev),
-                                                  avg ? static_cast<uint8_t*>(delta_wire_dev) : nullptr, main);
+    uint32_t* wire = static_cast<uint32_t*>(delta_wire_dev);
+    dlion_status st;
+    if (avg && wire != nullptr) {
+        st = dlion_aggregate(ctx, packed, wire, main);
+        if (st == DLION_OK) st = dlion_apply_delta(ctx, wire, x, main);
+    } else {
+        st = dlion_aggregate_apply(ctx, packed, x, wire, nullptr, main);
+    }
     if (st != DLION_OK) return st;
     if (host_delta_out != nullptr) {
-        const size_t bytes = avg ? static_cast<size_t>(ctx->d_pad) : words * 4;
-        if (cudaMemcpyAsync(host_delta_out, delta_wire_dev, bytes, cudaMemcpyDeviceToHost, main) != cudaSuccess) {
+        const size_t bytes = static_cast<size_t>(dlion_delta_planes(ctx)) * words * 4;
+        if (cudaMemcpyAsync(host_delta_out, wire, bytes, cudaMemcpyDeviceToHost, main) != cudaSuccess) {
             return DLION_ECUDA;
         }
     }
@@ -93,12 +118,13 @@ dlion_status dlion_aggregate(dlion_ctx* ctx, const uint32_t* packed, uint32_t* d
     dlion::WireParams p{};
     p.packed = packed;
     p.wire_out = delta_wire;
-    p.segs = ctx->segs_dev;
     p.tiles = ctx->tiles_dev;
-    p.nseg = ctx->nseg;
+    p.flat_d = 0;
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
     p.w_stride = ctx->d_pad / 32;
+    p.plane_stride = ctx->d_pad / 32;
+    p.kplanes = dlion_delta_planes(ctx);
     p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
     if (dlion::launch_wire(p, false, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
     if (ctx->ntiles != 0) ctx->launches += 1;
@@ -114,12 +140,13 @@ dlion_status dlion_apply_delta(dlion_ctx* ctx, const uint32_t* delta_wire, float
     dlion::WireParams p{};
     p.wire_in = delta_wire;
     p.x = x;
-    p.segs = ctx->segs_dev;
     p.tiles = ctx->tiles_dev;
-    p.nseg = ctx->nseg;
+    p.flat_d = 0;
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
     p.w_stride = ctx->d_pad / 32;
+    p.plane_stride = ctx->d_pad / 32;
+    p.kplanes = dlion_delta_planes(ctx);
     p.lr = ctx->lr;
     p.wd = ctx->wd;
     p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
@@ -165,15 +192,9 @@ const char* dlion_status_str(dlion_status s) {
 
 void dlion_destroy(dlion_ctx* ctx) {
     if (ctx == nullptr) return;
-    if (ctx->segs_dev != nullptr) cudaFree(ctx->segs_dev);
     if (ctx->tiles_dev != nullptr) cudaFree(ctx->tiles_dev);
     if (ctx->betas_dev != nullptr) cudaFree(ctx->betas_dev);
-    for (int k = 0; k < 2; ++k) {
-        if (ctx->copied[k] != nullptr) cudaEventDestroy(ctx->copied[k]);
-        if (ctx->consumed[k] != nullptr) cudaEventDestroy(ctx->consumed[k]);
-    }
-    if (ctx->entry != nullptr) cudaEventDestroy(ctx->entry);
-    if (ctx->copy_stream != nullptr) cudaStreamDestroy(ctx->copy_stream);
+    drop_pipeline(ctx);
     delete ctx;
 }
 

@@ -11,48 +11,18 @@
 // i is consumed.  HBM traffic per
 // coordinate: N (G + 8) + 8 B, G = gradient bytes (+ N/8 B with the wire buffer):
 // the 2 N/8 B round trip of the two-stage path is gone.
-#include "dlion_common.cuh"
+#include "worker_regs.cuh"
 
 namespace dlion {
 namespace {
 
 constexpr int kThreads = 256;             // 8 warps x 512 coordinates = one tile
-constexpr int kChunksPerWarp = 4;
 
 template <bool AVG>
 __device__ __forceinline__ float delta_of(uint32_t count, uint32_t thr, const float* avg_table) {
     if constexpr (AVG) return avg_table[count];
     return count >= thr ? 1.0f : -1.0f;
 }
-
-template <bool BF16>
-struct RawGrad4 { float4 v; };            // four gradients as stored
-template <>
-struct RawGrad4<true> { uint2 v; };
-
-template <bool BF16, bool MB16>
-struct WorkerRegs {                       // one worker's gradients and momenta of my coordinates
-    RawGrad4<BF16> g[kChunksPerWarp];
-    float4 m[kChunksPerWarp];
-    __device__ __forceinline__ void load(const FusedParams& p, unsigned long long at) {
-#pragma unroll
-        for (int u = 0; u < kChunksPerWarp; ++u) {
-            if constexpr (BF16) {
-                g[u].v = *(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(p.g) + at + u * kChunk));
-            } else {
-                g[u].v = *(reinterpret_cast<const float4*>(static_cast<const float*>(p.g) + at + u * kChunk));
-            }
-            m[u] = load_state4<MB16>(p.m, at + u * kChunk);
-        }
-    }
-    __device__ __forceinline__ float4 grad(int u) const {
-        if constexpr (BF16) {
-            return make_float4(bf16_lo(g[u].v.x), bf16_hi(g[u].v.x), bf16_lo(g[u].v.y), bf16_hi(g[u].v.y));
-        } else {
-            return g[u].v;
-        }
-    }
-};
 
 // Worker-side update of my coordinates for one worker: momenta stored, votes
 // added to cnt (one byte per coordinate), wire words written if requested.
@@ -138,7 +108,7 @@ step_fused_kernel(const __grid_constant__ FusedParams p) {
     const unsigned long long w_stride = p.d_pad / 32;
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.flat_d, tile);
         const uint32_t in_tile = warp * (kChunksPerWarp * kChunk);
         if (in_tile >= t.valid) continue;                          // warp-uniform
         const unsigned long long e0 = t.base + in_tile + lane * 4;  // my first coordinate (chunk 0)
@@ -155,12 +125,12 @@ step_fused_kernel(const __grid_constant__ FusedParams p) {
             }
             uint32_t* wire = p.packed == nullptr ? nullptr : p.packed + (t.base + in_tile) / 32;
             WorkerRegs<BF16, MB16> a, b;
-            a.load(p, e0);
+            a.load(p.g, p.m, e0);
             uint32_t i = 0;
             for (; i + 2 <= n; i += 2) {
-                b.load(p, (i + 1) * p.d_pad + e0);
+                b.load(p.g, p.m, (i + 1) * p.d_pad + e0);
                 consume<BF16, MB16>(p, a, i, i * p.d_pad + e0, wire == nullptr ? nullptr : wire + i * w_stride, lane, cnt);
-                if (i + 2 < n) a.load(p, (i + 2) * p.d_pad + e0);
+                if (i + 2 < n) a.load(p.g, p.m, (i + 2) * p.d_pad + e0);
                 consume<BF16, MB16>(p, b, i + 1, (i + 1) * p.d_pad + e0, wire == nullptr ? nullptr : wire + (i + 1) * w_stride,
                               lane, cnt);
             }

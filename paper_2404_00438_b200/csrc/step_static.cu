@@ -6,12 +6,18 @@
 // where cudaMalloc's implicit device synchronisation is not acceptable, or a
 // plug-in that is only allowed to use the buffers it was given.  The regular
 // path needs two pieces of device memory besides the caller's tensors: the
-// context's segment table (allocated by dlion_init) and the 1-bit wire buffer
-// between the two kernels.  Here both live in a fixed array that is part of the
-// library image, so the call needs neither dlion_init nor a wire buffer.
+// context's tile table (allocated by dlion_init) and the 1-bit wire buffer
+// between the two kernels.  Here the wire buffer is a fixed array that is part
+// of the library image and the parameters are a flat vector, which needs no
+// table, so the call needs neither dlion_init nor a caller-supplied wire buffer.
 //
-// The price: the array has a fixed size, every GPU that loads the library holds
-// it until the process exits, and all calls on a device share it.
+// The price: the array has a fixed size, every GPU on which the library's
+// device code gets loaded holds it until the process exits, and all calls on a
+// device share it.  The FIRST call on a device is a set-up call: it makes the
+// CUDA runtime load this library's device code (which is when the array is
+// reserved) and looks up the array's address.  Make it at start-up, before
+// another allocator takes the remaining memory and before any stream capture;
+// only the calls after it allocate nothing.
 #include <mutex>
 
 #include "dlion_common.cuh"
@@ -20,12 +26,11 @@
 namespace {
 
 constexpr unsigned long long kMaxCoordWorkers = DLION_STATIC_MAX_COORD_WORKERS;   // N * d_pad limit
-constexpr size_t kHeaderWords = 64;                               // 256 B: the one-row segment table
 constexpr size_t kWireWords = kMaxCoordWorkers / 32;              // 16 MiB of sign bits
 
 // Scratch shared by every dlion_step_static call on this device.  In host code
 // this name is only a handle for cudaGetSymbolAddress, never a device pointer.
-static __device__ __align__(256) uint32_t g_static_scratch[kHeaderWords + kWireWords];
+static __device__ __align__(256) uint32_t g_static_scratch[kWireWords];
 
 constexpr int kMaxDevices = 64;
 struct PerDevice {
@@ -53,13 +58,6 @@ cudaError_t setup_device(int dev, PerDevice* out) {
     return cudaSuccess;
 }
 
-// Writes the one-row segment table of a flat vector into the scratch header.
-__global__ void write_flat_row_kernel(dlion::SegDev* row, unsigned long long d) {
-    row->elem_offset = 0;
-    row->numel = d;
-    row->first_tile = 0;
-}
-
 using dlion::aligned16;
 using dlion::nonneg_finite;
 using dlion::unit_interval;
@@ -71,7 +69,7 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
                                           dlion_gdtype gdtype, const void* grads, float* m, float* x,
                                           void* cuda_stream) {
     if (d == 0 || grads == nullptr || m == nullptr || x == nullptr) return DLION_EINVAL;
-    if (n_workers == 0 || n_workers > DLION_MAX_WORKERS_BYTE_COUNTS) return DLION_EINVAL;
+    if (n_workers == 0 || n_workers > DLION_MAX_WORKERS) return DLION_EINVAL;
     if (!unit_interval(beta1) || !unit_interval(beta2)) return DLION_EINVAL;
     if (!nonneg_finite(lr) || !nonneg_finite(weight_decay)) return DLION_EINVAL;
     if (mode != DLION_MAJORITY && mode != DLION_AVERAGE) return DLION_EINVAL;
@@ -88,24 +86,18 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
     if (setup_device(dev, &pd) != cudaSuccess) return DLION_ECUDA;
 
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    dlion::SegDev* row = reinterpret_cast<dlion::SegDev*>(pd.scratch);
-    uint32_t* wire = pd.scratch + kHeaderWords;
+    uint32_t* wire = pd.scratch;
     const unsigned long long ntiles = (d + dlion::kTile - 1) / dlion::kTile;
 
-    // The header keeps the previous call's row: rewrite it.  The wire buffer keeps
-    // the previous call's bits: the worker-side kernel overwrites every word that
-    // holds a parameter and the server-side kernel reads no other word, so
-    // nothing has to be cleared.
-    write_flat_row_kernel<<<1, 1, 0, s>>>(row, d);
-    if (cudaGetLastError() != cudaSuccess) return DLION_ECUDA;
-
+    // The wire buffer keeps the previous call's bits: the worker-side kernel
+    // overwrites every word that holds a parameter and the server-side kernel reads
+    // no other word, so nothing has to be cleared.
     dlion::WorkerParams wp;
     wp.g = grads;
     wp.m = m;
     wp.packed = wire;
-    wp.segs = row;
     wp.tiles = nullptr;
-    wp.nseg = 1;
+    wp.flat_d = d;
     wp.n_workers = n_workers;
     wp.ntiles = ntiles;
     wp.d_pad = d_pad;
@@ -125,9 +117,8 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
     ap.x = x;
     ap.delta_bits = nullptr;
     ap.count = nullptr;
-    ap.segs = row;
     ap.tiles = nullptr;
-    ap.nseg = 1;
+    ap.flat_d = d;
     ap.n_workers = n_workers;
     ap.ntiles = ntiles;
     ap.w_stride = d_pad / 32;

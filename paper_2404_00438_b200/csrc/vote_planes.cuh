@@ -2,6 +2,8 @@
 // one 32-coordinate word position; plane p holds bit p of the 32 vote counts.
 #pragma once
 
+#include <type_traits>
+
 #include "dlion_common.cuh"
 
 namespace dlion {
@@ -103,53 +105,113 @@ __device__ __forceinline__ uint32_t planes_ge(const uint32_t (&pl)[kMaxPlanes], 
     return gt | eq;
 }
 
-// Votes of my four coordinates in chunk c: the Delta bits (dn, bit q = coordinate q)
-// and, when counts are needed, the four vote counts.  Up to 8 planes the counts are
-// packed one per byte in lo; beyond (N > 255) two 16-bit counts each in lo and hi.
-struct Votes4 {
-    uint32_t dn, lo, hi;
+// ---- from bit planes to per-coordinate counts -------------------------------
+//
+// The lane that owns a word holds its 32 vote counts as bit planes; the lanes that
+// update x need them per coordinate.  The owner turns planes 0..7 into bytes with
+// three rounds of word-wide delta swaps (an 8x8 bit-matrix transpose of each
+// byte column: about 60 logic ops for all 32 coordinates, fewer when upper planes
+// are known to be zero) and publishes them in shared memory; a consumer then needs
+// one 16-byte load and one byte permute per coordinate.
+//
+// After the transpose, register c holds in byte k the count of coordinate 8k + c.
+
+__device__ __forceinline__ void delta_swap(uint32_t& a, uint32_t& b, uint32_t mask, int s) {
+    const uint32_t t = ((a >> s) ^ b) & mask;      // a's upper field <-> b's lower field
+    b ^= t;
+    a ^= t << s;
+}
+
+template <int PLANES, int P0>
+__device__ __forceinline__ void planes_to_bytes(const uint32_t (&pl)[kMaxPlanes], uint32_t (&r)[8]) {
+#pragma unroll
+    for (int p = 0; p < 8; ++p) r[p] = (P0 + p < PLANES) ? pl[P0 + p] : 0u;
+#pragma unroll
+    for (int p = 0; p < 4; ++p) delta_swap(r[p], r[p + 4], 0x0F0F0F0Fu, 4);
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+        if ((p & 2) == 0) delta_swap(r[p], r[p + 2], 0x33333333u, 2);
+    }
+#pragma unroll
+    for (int p = 0; p < 8; p += 2) delta_swap(r[p], r[p + 1], 0x55555555u, 1);
+}
+
+// One warp's hand-off area.  half[h][o] = registers 4h..4h+3 of owner lane o; the
+// spare 33rd slot shifts the second half by four banks, so the two halves a
+// quarter-warp reads together never collide.
+struct CountSlots {
+    uint4 half[2][33];
 };
 
-// All 32 lanes must call this together.
-template <int PLANES, bool COUNTS>
-__device__ __forceinline__ Votes4 my_votes(const uint32_t (&pl)[kMaxPlanes], uint32_t dword, int c, uint32_t lane) {
-    const uint32_t src = 4u * c + (lane >> 3);           // lane that owns my word
-    const uint32_t sh = 4u * (lane & 7u);
-    Votes4 v;
-    v.dn = (__shfl_sync(kFull, dword, src) >> sh) & 0xFu;
-    v.lo = 0;
-    v.hi = 0;
-    if constexpr (COUNTS) {
-#pragma unroll
-        for (int q = 0; q < PLANES; ++q) {
-            const uint32_t nib = (__shfl_sync(kFull, pl[q], src) >> sh) & 0xFu;
-            if constexpr (PLANES <= 8) {
-                v.lo += spread_nibble(nib) << q;
-            } else {
-                v.lo += ((nib & 1u) | ((nib & 2u) << 15)) << q;
-                v.hi += (((nib >> 2) & 1u) | ((nib & 8u) << 13)) << q;
-            }
-        }
+template <bool WIDE>
+struct CountArea {                                  // N > 255: bits 8..15 of every count too
+    CountSlots lo, hi;
+};
+template <>
+struct CountArea<false> {
+    CountSlots lo;
+};
+
+// Owner side: all 32 lanes call this together, once per tile, after the vote.
+template <int PLANES>
+__device__ __forceinline__ void publish_counts(const uint32_t (&pl)[kMaxPlanes], CountArea<(PLANES > 8)>* area,
+                                               uint32_t lane) {
+    __syncwarp();                                   // the previous tile's readers are done
+    uint32_t r[8];
+    planes_to_bytes<PLANES, 0>(pl, r);
+    area->lo.half[0][lane] = make_uint4(r[0], r[1], r[2], r[3]);
+    area->lo.half[1][lane] = make_uint4(r[4], r[5], r[6], r[7]);
+    if constexpr (PLANES > 8) {
+        planes_to_bytes<PLANES, 8>(pl, r);
+        area->hi.half[0][lane] = make_uint4(r[0], r[1], r[2], r[3]);
+        area->hi.half[1][lane] = make_uint4(r[4], r[5], r[6], r[7]);
     }
-    return v;
+    __syncwarp();
 }
+
+// Consumer side: the vote counts of my four coordinates in chunk c (coordinates
+// 128c + 4*lane .. +3 of the warp's 1024): they sit in word 4c + lane/8, at in-word
+// positions 4*(lane%8) + q, i.e. registers 4*(lane%2) + q, byte (lane%8)/2.
+struct Counts4 {
+    uint32_t c[4];
+};
 
 template <int PLANES>
-__device__ __forceinline__ uint32_t count_of(const Votes4& v, int q) {
-    if constexpr (PLANES <= 8) return (v.lo >> (8 * q)) & 0xFFu;
-    return ((q < 2 ? v.lo : v.hi) >> (16 * (q & 1))) & 0xFFFFu;
+__device__ __forceinline__ Counts4 my_counts(const CountArea<(PLANES > 8)>* area, int c, uint32_t lane) {
+    const uint32_t owner = 4u * c + (lane >> 3);
+    const uint32_t sel = 0x4440u | ((lane & 7u) >> 1);            // byte k of the first operand, then zeros
+    const uint4 v = area->lo.half[lane & 1u][owner];
+    Counts4 k;
+    k.c[0] = __byte_perm(v.x, 0u, sel);
+    k.c[1] = __byte_perm(v.y, 0u, sel);
+    k.c[2] = __byte_perm(v.z, 0u, sel);
+    k.c[3] = __byte_perm(v.w, 0u, sel);
+    if constexpr (PLANES > 8) {
+        const uint4 h = area->hi.half[lane & 1u][owner];
+        k.c[0] |= __byte_perm(h.x, 0u, sel) << 8;
+        k.c[1] |= __byte_perm(h.y, 0u, sel) << 8;
+        k.c[2] |= __byte_perm(h.z, 0u, sel) << 8;
+        k.c[3] |= __byte_perm(h.w, 0u, sel) << 8;
+    }
+    return k;
 }
 
-// Delta of coordinate q.  Averaging: from the per-warp table while the counts fit
-// it (N <= 255), else the correctly rounded quotient directly.
+// The Delta bits of my four coordinates in chunk c, from the owner's Delta word
+// (Majority Vote when no counts are needed).  All 32 lanes must call this together.
+__device__ __forceinline__ uint32_t my_delta_bits(uint32_t dword, int c, uint32_t lane) {
+    return (__shfl_sync(kFull, dword, 4u * c + (lane >> 3)) >> (4u * (lane & 7u))) & 0xFu;
+}
+
+// Delta of a coordinate from its vote count P.  Majority Vote: +1 iff P >= ceil(N/2).
+// Averaging: from the per-warp table while the counts fit it (N <= 255), else the
+// correctly rounded quotient directly.
 template <int PLANES, bool AVG>
-__device__ __forceinline__ float delta_value(const Votes4& v, int q, const float* avg_table, uint32_t n) {
+__device__ __forceinline__ float delta_of_count(uint32_t count, uint32_t thr, const float* avg_table, uint32_t n) {
     if constexpr (AVG) {
-        const uint32_t c = count_of<PLANES>(v, q);
-        if constexpr (PLANES <= 8) return avg_table[c];
-        return __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)), static_cast<float>(n));
+        if constexpr (PLANES <= 8) return avg_table[count];
+        return __fdiv_rn(static_cast<float>(2 * static_cast<int>(count) - static_cast<int>(n)), static_cast<float>(n));
     }
-    return ((v.dn >> q) & 1u) ? 1.0f : -1.0f;
+    return count >= thr ? 1.0f : -1.0f;
 }
 
 // Fills a warp's private table of Averaging's Delta for every count (N <= 255 only).
@@ -161,6 +223,25 @@ __device__ __forceinline__ void fill_avg_table(float* avg_table, uint32_t n, uin
                                      static_cast<float>(n));
         }
         __syncwarp();
+    }
+}
+
+// Plane capacities the kernels are compiled for: the exact plane count up to 8
+// (N <= 255, where the count matters for speed), then 12 and 16.  A capacity
+// above the needed count only adds zero planes.
+template <typename F>
+inline cudaError_t dispatch_planes(uint32_t n_workers, F&& f) {
+    switch (planes_for(n_workers)) {
+        case 1: return f(std::integral_constant<int, 1>{});
+        case 2: return f(std::integral_constant<int, 2>{});
+        case 3: return f(std::integral_constant<int, 3>{});
+        case 4: return f(std::integral_constant<int, 4>{});
+        case 5: return f(std::integral_constant<int, 5>{});
+        case 6: return f(std::integral_constant<int, 6>{});
+        case 7: return f(std::integral_constant<int, 7>{});
+        case 8: return f(std::integral_constant<int, 8>{});
+        case 9: case 10: case 11: case 12: return f(std::integral_constant<int, 12>{});
+        default: return f(std::integral_constant<int, 16>{});
     }
 }
 

@@ -21,6 +21,7 @@ namespace dlion {
 namespace {
 
 constexpr int kThreads = 128;             // 4 warps x 1024 coordinates = one tile
+constexpr int kWarps = kThreads / 32;
 
 template <int PLANES, bool AVG>
 __global__ void __launch_bounds__(kThreads)
@@ -29,7 +30,7 @@ aggregate_kernel(const __grid_constant__ WireParams p) {
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t thr = (p.n_workers + 1u) >> 1;
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.flat_d, tile);
         const uint32_t my0 = warp * kWarpSpan + lane * 32;          // first coordinate of my word
         if (my0 >= t.valid) continue;                               // my word holds no parameter
         const uint32_t nbits = t.valid - my0 >= 32u ? 32u : t.valid - my0;
@@ -39,7 +40,9 @@ aggregate_kernel(const __grid_constant__ WireParams p) {
         count_votes<PLANES>(pl, p.packed + word_idx, p.w_stride, p.n_workers, true);
         if constexpr (AVG) {
 #pragma unroll
-            for (int q = 0; q < PLANES; ++q) p.wire_out[q * p.w_stride + word_idx] = pl[q] & vmask;
+            for (int q = 0; q < PLANES; ++q) {
+                if (q < static_cast<int>(p.kplanes)) p.wire_out[q * p.plane_stride + word_idx] = pl[q] & vmask;
+            }
         } else {
             p.wire_out[word_idx] = planes_ge<PLANES>(pl, thr) & vmask;
         }
@@ -49,15 +52,17 @@ aggregate_kernel(const __grid_constant__ WireParams p) {
 template <int PLANES, bool AVG>
 __global__ void __launch_bounds__(kThreads, 6)
 apply_delta_kernel(const __grid_constant__ WireParams p) {
-    __shared__ float avg_tables[(AVG && PLANES <= 8) ? kThreads / 32 : 1][(AVG && PLANES <= 8) ? 256 : 1];
+    __shared__ float avg_tables[(AVG && PLANES <= 8) ? kWarps : 1][(AVG && PLANES <= 8) ? 256 : 1];
+    __shared__ CountArea<(PLANES > 8)> areas[AVG ? kWarps : 1];
     const uint32_t n = p.n_workers;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
     float* avg_table = avg_tables[(AVG && PLANES <= 8) ? warp : 0];
+    CountArea<(PLANES > 8)>* area = &areas[AVG ? warp : 0];
     bool have_table = !AVG;
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.flat_d, tile);
         const uint32_t w0 = warp * kWarpSpan;
         if (w0 >= t.valid) continue;                                // warp-uniform
         const bool full = w0 + kWarpSpan <= t.valid;
@@ -70,34 +75,47 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) xv[c] = *(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
         }
-        uint32_t pl[kMaxPlanes];
         uint32_t dword = 0;
         if constexpr (AVG) {
+            uint32_t pl[kMaxPlanes];
 #pragma unroll
-            for (int q = 0; q < PLANES; ++q) pl[q] = live ? __ldg(p.wire_in + q * p.w_stride + word_idx) : 0u;
+            for (int q = 0; q < kMaxPlanes; ++q) {
+                pl[q] = (q < PLANES && q < static_cast<int>(p.kplanes) && live)
+                            ? __ldg(p.wire_in + q * p.plane_stride + word_idx) : 0u;
+            }
+            if (!have_table) {
+                fill_avg_table<PLANES>(avg_table, n, lane);
+                have_table = true;
+            }
+            publish_counts<PLANES>(pl, area, lane);
         } else {
             dword = live ? __ldg(p.wire_in + word_idx) : 0u;
         }
-        if (!have_table) {
-            fill_avg_table<PLANES>(avg_table, n, lane);
-            have_table = true;
-        }
 #pragma unroll
         for (int c = 0; c < 8; ++c) {
-            const Votes4 vt = my_votes<PLANES, AVG>(pl, dword, c, lane);
+            float d[4];
+            if constexpr (AVG) {
+                const Counts4 k = my_counts<PLANES>(area, c, lane);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) d[q] = delta_of_count<PLANES, true>(k.c[q], 0u, avg_table, n);
+            } else {
+                const uint32_t dn = my_delta_bits(dword, c, lane);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) d[q] = ((dn >> q) & 1u) ? 1.0f : -1.0f;
+            }
             const uint32_t j0 = w0 + c * kChunk + lane * 4;
             if (j0 >= t.valid) continue;                            // after the shuffles: all lanes took part
             const unsigned long long e = xe + c * kChunk;
             if (full) {
                 float4 v = xv[c];
-                v.x = apply_coord(v.x, delta_value<PLANES, AVG>(vt, 0, avg_table, n), p.lr, p.wd);
-                v.y = apply_coord(v.y, delta_value<PLANES, AVG>(vt, 1, avg_table, n), p.lr, p.wd);
-                v.z = apply_coord(v.z, delta_value<PLANES, AVG>(vt, 2, avg_table, n), p.lr, p.wd);
-                v.w = apply_coord(v.w, delta_value<PLANES, AVG>(vt, 3, avg_table, n), p.lr, p.wd);
+                v.x = apply_coord(v.x, d[0], p.lr, p.wd);
+                v.y = apply_coord(v.y, d[1], p.lr, p.wd);
+                v.z = apply_coord(v.z, d[2], p.lr, p.wd);
+                v.w = apply_coord(v.w, d[3], p.lr, p.wd);
                 *reinterpret_cast<float4*>(p.x + e) = v;
             } else {
                 for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
-                    p.x[e + q] = apply_coord(p.x[e + q], delta_value<PLANES, AVG>(vt, q, avg_table, n), p.lr, p.wd);
+                    p.x[e + q] = apply_coord(p.x[e + q], d[q], p.lr, p.wd);
                 }
             }
         }
@@ -127,24 +145,7 @@ uint32_t planes_for(uint32_t n_workers) {      // bit length of N = ceil(log2(N+
 }
 
 cudaError_t launch_wire(const WireParams& p, bool apply, cudaStream_t s) {
-    switch (planes_for(p.n_workers)) {
-        case 1: return launch<1>(p, apply, s);
-        case 2: return launch<2>(p, apply, s);
-        case 3: return launch<3>(p, apply, s);
-        case 4: return launch<4>(p, apply, s);
-        case 5: return launch<5>(p, apply, s);
-        case 6: return launch<6>(p, apply, s);
-        case 7: return launch<7>(p, apply, s);
-        case 8: return launch<8>(p, apply, s);
-        case 9: return launch<9>(p, apply, s);
-        case 10: return launch<10>(p, apply, s);
-        case 11: return launch<11>(p, apply, s);
-        case 12: return launch<12>(p, apply, s);
-        case 13: return launch<13>(p, apply, s);
-        case 14: return launch<14>(p, apply, s);
-        case 15: return launch<15>(p, apply, s);
-        default: return launch<16>(p, apply, s);
-    }
+    return dispatch_planes(p.n_workers, [&](auto planes) { return launch<decltype(planes)::value>(p, apply, s); });
 }
 
 }  // namespace dlion

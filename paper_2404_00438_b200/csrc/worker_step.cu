@@ -36,7 +36,7 @@ worker_step_kernel(const WorkerParams p) {
     const unsigned long long worker = blockIdx.y;                  // grid: x = tile (fastest), y = worker
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
-        const TileRef t = find_tile(p.tiles, p.segs, p.nseg, tile);
+        const TileRef t = find_tile(p.tiles, p.flat_d, tile);
         const unsigned long long wbase = worker * p.d_pad;         // element offset of this worker
         const Betas k = betas_of(p.betas, p.k, p.worker0 + worker);
         const uint32_t in_tile = warp * (kChunksPerWarp * kChunk); // first coordinate of this warp

@@ -25,7 +25,7 @@ OK, EINVAL, EALIGN, ENOMEM, ECUDA, ESTATE = range(6)
 EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_set_momentum_dtype",
            "dlion_set_worker_betas", "dlion_worker_step",
            "dlion_aggregate_apply", "dlion_aggregate", "dlion_apply_delta", "dlion_delta_planes",
-           "dlion_step_fused", "dlion_step_host", "dlion_step_static",
+           "dlion_step_fused", "dlion_step_global", "dlion_step_host", "dlion_step_static",
            "dlion_wire_bytes",
            "dlion_launch_count", "dlion_status_str", "dlion_destroy")
 
@@ -71,6 +71,8 @@ def _load() -> ctypes.CDLL:
     lib.dlion_delta_planes.restype = u32
     lib.dlion_step_fused.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.dlion_step_fused.restype = i32
+    lib.dlion_step_global.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.dlion_step_global.restype = i32
     lib.dlion_step_host.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.dlion_step_host.restype = i32
     lib.dlion_step_static.argtypes = [u64, u32, f32, f32, f32, f32, i32, i32, vp, vp, vp, vp]
@@ -120,6 +122,12 @@ def step_static(d: int, n_workers: int, beta1: float, beta2: float, lr: float, w
     allocate device memory (no context, no wire buffer: both live in a fixed array inside the
     library, shared by all calls on the device).  Raises DlionError when N * d_pad exceeds
     STATIC_MAX_COORD_WORKERS."""
+    d_pad = (int(d) + ALIGN - 1) // ALIGN * ALIGN
+    dev = torch.cuda.current_device() if torch.cuda.is_available() else None
+    fits = 0 < int(n_workers) * d_pad <= STATIC_MAX_COORD_WORKERS      # else the library rejects the size itself
+    check_tensor(grads, "grads", _GRAD_DTYPES.get(int(gdtype)), int(n_workers) * d_pad if fits else 0, dev)
+    check_tensor(m, "m", (torch.float32,), int(n_workers) * d_pad if fits else 0, dev)
+    check_tensor(x, "x", (torch.float32,), d_pad if fits else 0, dev)
     st = _lib.dlion_step_static(int(d), int(n_workers), beta1, beta2, lr, weight_decay, int(mode),
                                 int(gdtype), _ptr(grads), _ptr(m), _ptr(x), _stream())
     if st != OK:
@@ -134,6 +142,40 @@ def _stream() -> int:
     return torch.cuda.current_stream().cuda_stream
 
 
+_WORD_DTYPES = tuple(t for t in (torch.int32, getattr(torch, "uint32", None)) if t is not None)
+_GRAD_DTYPES = {GRAD_F32: (torch.float32,), GRAD_BF16: (torch.bfloat16,)}
+_STATE_DTYPES = {STATE_F32: (torch.float32,), STATE_BF16: (torch.bfloat16,)}
+
+
+def check_tensor(t: Optional[torch.Tensor], name: str, dtypes, min_numel: int,
+                 device_index: Optional[int], optional: bool = False, host: bool = False) -> None:
+    """Raises ValueError unless ``t`` can be handed to the C ABI as a raw pointer: on the
+    context's GPU (or, with ``host``, in host memory), contiguous, of one of ``dtypes`` and
+    holding at least ``min_numel`` elements.  The C side sees only an address, so a wrong
+    size, a strided view or a tensor on another device would otherwise become an
+    out-of-bounds access inside a kernel.  Nothing is launched when this raises."""
+    if t is None:
+        if optional:
+            return
+        raise ValueError(f"{name}: a tensor is required")
+    if not isinstance(t, torch.Tensor):
+        raise ValueError(f"{name}: expected a torch.Tensor, got {type(t).__name__}")
+    if host:
+        if t.is_cuda:
+            raise ValueError(f"{name}: must be in host memory")
+    else:
+        if not t.is_cuda:
+            raise ValueError(f"{name}: must be a CUDA tensor (the library has no CPU path)")
+        if device_index is not None and t.device.index != device_index:
+            raise ValueError(f"{name}: is on cuda:{t.device.index}, the context lives on cuda:{device_index}")
+    if dtypes is not None and t.dtype not in dtypes:
+        raise ValueError(f"{name}: dtype {t.dtype}, expected one of {tuple(dtypes)}")
+    if not t.is_contiguous():
+        raise ValueError(f"{name}: must be contiguous (got strides {tuple(t.stride())})")
+    if t.numel() < min_numel:
+        raise ValueError(f"{name}: {t.numel()} elements, the call reads or writes {min_numel}")
+
+
 class Dlion:
     """Owner of one ``dlion_ctx``.  Methods mirror the C calls one to one."""
 
@@ -146,17 +188,24 @@ class Dlion:
         if st != OK:
             self._ctx = ctypes.c_void_p()
             raise DlionError(st, "dlion_init")
-        self.d_pad, self.n_workers, self.mode, self.gdtype = int(d_pad), int(n_workers), mode, gdtype
+        self.d_pad, self.n_workers, self.mode, self.gdtype = int(d_pad), int(n_workers), int(mode), int(gdtype)
+        self.sdtype = STATE_F32
+        self.words = self.d_pad // 32
+        self.device_index = torch.cuda.current_device()
 
     def _check(self, st: int, where: str) -> None:
         if st != OK:
             raise DlionError(st, where)
+
+    def _t(self, t, name, dtypes, min_numel, optional=False, host=False) -> None:
+        check_tensor(t, name, dtypes, min_numel, self.device_index, optional=optional, host=host)
 
     def set_lr(self, lr: float) -> None:
         self._check(_lib.dlion_set_lr(self._ctx, lr), "dlion_set_lr")
 
     def set_momentum_dtype(self, sdtype: int) -> None:
         self._check(_lib.dlion_set_momentum_dtype(self._ctx, int(sdtype)), "dlion_set_momentum_dtype")
+        self.sdtype = int(sdtype)
 
     def set_worker_betas(self, worker: int, beta1: float, beta2: float) -> None:
         self._check(_lib.dlion_set_worker_betas(self._ctx, int(worker), beta1, beta2),
@@ -164,20 +213,32 @@ class Dlion:
 
     def worker_step(self, worker: int, grads: torch.Tensor, m: torch.Tensor,
                     packed: torch.Tensor) -> None:
+        k = self.n_workers if int(worker) < 0 else 1
+        self._t(grads, "grads", _GRAD_DTYPES[self.gdtype], k * self.d_pad)
+        self._t(m, "m", _STATE_DTYPES[self.sdtype], k * self.d_pad)
+        self._t(packed, "packed", _WORD_DTYPES, k * self.words)
         self._check(_lib.dlion_worker_step(self._ctx, int(worker), _ptr(grads), _ptr(m), _ptr(packed),
                                            _stream()), "dlion_worker_step")
 
     def aggregate_apply(self, packed: torch.Tensor, x: torch.Tensor,
                         delta_bits_out: Optional[torch.Tensor] = None,
                         count_out: Optional[torch.Tensor] = None) -> None:
+        self._t(packed, "packed", _WORD_DTYPES, self.n_workers * self.words)
+        self._t(x, "x", (torch.float32,), self.d_pad)
+        self._t(delta_bits_out, "delta_bits_out", _WORD_DTYPES, self.words, optional=True)
+        self._t(count_out, "count_out", (torch.uint8,), self.d_pad, optional=True)
         self._check(_lib.dlion_aggregate_apply(self._ctx, _ptr(packed), _ptr(x), _ptr(delta_bits_out),
                                                _ptr(count_out), _stream()), "dlion_aggregate_apply")
 
     def aggregate(self, packed: torch.Tensor, delta_wire: torch.Tensor) -> None:
+        self._t(packed, "packed", _WORD_DTYPES, self.n_workers * self.words)
+        self._t(delta_wire, "delta_wire", _WORD_DTYPES, self.delta_planes() * self.words)
         self._check(_lib.dlion_aggregate(self._ctx, _ptr(packed), _ptr(delta_wire), _stream()),
                     "dlion_aggregate")
 
     def apply_delta(self, delta_wire: torch.Tensor, x: torch.Tensor) -> None:
+        self._t(delta_wire, "delta_wire", _WORD_DTYPES, self.delta_planes() * self.words)
+        self._t(x, "x", (torch.float32,), self.d_pad)
         self._check(_lib.dlion_apply_delta(self._ctx, _ptr(delta_wire), _ptr(x), _stream()),
                     "dlion_apply_delta")
 
@@ -186,13 +247,36 @@ class Dlion:
 
     def step_fused(self, grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor,
                    packed_out: Optional[torch.Tensor] = None) -> None:
+        self._t(grads, "grads", _GRAD_DTYPES[self.gdtype], self.n_workers * self.d_pad)
+        self._t(m, "m", _STATE_DTYPES[self.sdtype], self.n_workers * self.d_pad)
+        self._t(x, "x", (torch.float32,), self.d_pad)
+        self._t(packed_out, "packed_out", _WORD_DTYPES, self.n_workers * self.words, optional=True)
         self._check(_lib.dlion_step_fused(self._ctx, _ptr(grads), _ptr(m), _ptr(x), _ptr(packed_out),
                                           _stream()), "dlion_step_fused")
+
+    def step_global(self, grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor,
+                    delta_bits_out: Optional[torch.Tensor] = None) -> None:
+        self._t(grads, "grads", _GRAD_DTYPES[self.gdtype], self.n_workers * self.d_pad)
+        self._t(m, "m", (torch.float32,), self.n_workers * self.d_pad)
+        self._t(x, "x", (torch.float32,), self.d_pad)
+        self._t(delta_bits_out, "delta_bits_out", _WORD_DTYPES, self.words, optional=True)
+        self._check(_lib.dlion_step_global(self._ctx, _ptr(grads), _ptr(m), _ptr(x), _ptr(delta_bits_out),
+                                           _stream()), "dlion_step_global")
 
     def step_host(self, host_grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor,
                   packed: torch.Tensor, staging: torch.Tensor,
                   delta_wire_dev: Optional[torch.Tensor] = None,
                   host_delta_out: Optional[torch.Tensor] = None) -> None:
+        wire_bytes = self.delta_planes() * self.words * 4
+        self._t(host_grads, "host_grads", _GRAD_DTYPES[self.gdtype], self.n_workers * self.d_pad, host=True)
+        self._t(m, "m", _STATE_DTYPES[self.sdtype], self.n_workers * self.d_pad)
+        self._t(x, "x", (torch.float32,), self.d_pad)
+        self._t(packed, "packed", _WORD_DTYPES, self.n_workers * self.words)
+        self._t(staging, "staging", _GRAD_DTYPES[self.gdtype], 2 * self.d_pad)
+        for t, name, host in ((delta_wire_dev, "delta_wire_dev", False), (host_delta_out, "host_delta_out", True)):
+            self._t(t, name, None, 0, optional=True, host=host)
+            if t is not None and t.numel() * t.element_size() < wire_bytes:
+                raise ValueError(f"{name}: {t.numel() * t.element_size()} bytes, the message has {wire_bytes}")
         self._check(_lib.dlion_step_host(self._ctx, _ptr(host_grads), _ptr(m), _ptr(x), _ptr(packed),
                                          _ptr(staging), _ptr(delta_wire_dev), _ptr(host_delta_out),
                                          _stream()), "dlion_step_host")

@@ -215,21 +215,24 @@ def _scalar(v: float, device) -> torch.Tensor:
 
 
 def fill_grads(w: Workload, step: int, out: torch.Tensor, lo: int = 0,
-               hi: Optional[int] = None) -> torch.Tensor:
+               hi: Optional[int] = None, workers: Optional[Sequence[int]] = None) -> torch.Tensor:
     """Write g_{i,step}[lo:hi] for every worker into ``out`` ([N, hi-lo], f32 or bf16).
 
     ``lo``/``hi`` are arena indices (padding included); padding lanes get 0.
+    ``workers`` restricts the rows to those workers (``out`` is [len(workers), hi-lo]);
+    a worker's values do not depend on which other workers are generated with it.
     """
     hi = w.d_pad if hi is None else hi
     dev = out.device
-    assert out.shape == (w.n_workers, hi - lo)
+    ids = list(range(w.n_workers)) if workers is None else [int(i) for i in workers]
+    assert out.shape == (len(ids), hi - lo)
     a_s, a_p, sc = (_scalar(v, dev) for v in (w.a_shared, w.a_private, w.scale))
     zthr = int(round(w.zero_frac * 0.5 * 65536))
     for c0 in range(lo, hi, _CHUNK):
         c1 = min(hi, c0 + _CHUNK)
         s, s_bits = _normal_and_bits(_key(w.seed, step, 0), c0, c1, dev)
         s = s * a_s
-        for i in range(w.n_workers):
+        for row, i in enumerate(ids):
             e, e_bits = _normal_and_bits(_key(w.seed, step, 1 + i), c0, c1, dev)
             g = e * a_p
             g = g + s
@@ -237,7 +240,7 @@ def fill_grads(w: Workload, step: int, out: torch.Tensor, lo: int = 0,
                 g = g * sc
             if zthr:
                 g = torch.where((s_bits < zthr) | (e_bits < zthr), torch.zeros_like(g), g)
-            out[i, c0 - lo:c1 - lo] = g.to(out.dtype)
+            out[row, c0 - lo:c1 - lo] = g.to(out.dtype)
     _zero_padding(w, out, lo, hi)
     return out
 

@@ -133,9 +133,16 @@ def test_argument_errors_with_a_context(dl):
     with pytest.raises(dl.DlionError) as e:
         ctx.aggregate_apply(packed, x[1:])           # 4-byte aligned only
     assert e.value.status == dl.EALIGN
+    g_big = torch.zeros(2 * w.d_pad + 4, device=dev)
     with pytest.raises(dl.DlionError) as e:
-        ctx.worker_step(-1, g.view(-1)[1:], m, packed)
+        ctx.worker_step(-1, g_big[1:], m, packed)     # long enough and contiguous, but 4-byte aligned only
     assert e.value.status == dl.EALIGN
+    with pytest.raises(ValueError):                  # too short: refused by the binding, nothing launched
+        ctx.worker_step(-1, g.view(-1)[1:], m, packed)
+    with pytest.raises(ValueError):                  # one worker's slice passed for all workers
+        ctx.worker_step(-1, g[0], m, packed)
+    with pytest.raises(ValueError):                  # strided view
+        ctx.aggregate_apply(packed[:, 8:40], x)
     raw = dl.lib()
     assert raw.dlion_worker_step(ctx._ctx, -1, None, m.data_ptr(), packed.data_ptr(), None) == dl.EINVAL
     assert raw.dlion_step_host(ctx._ctx, g.data_ptr(), m.data_ptr(), x.data_ptr(), packed.data_ptr(),
@@ -147,8 +154,10 @@ def test_argument_errors_with_a_context(dl):
 
 # ---------------------------------------------------------------- host-gradient step
 @pytest.mark.parametrize("mode", [MAJ, AVG])
-def test_step_host_matches_oracle(dl, mode):
-    w = inputs.custom([70000, 333], 5, mode, "bf16", scale=1e-3, lr=1e-3, weight_decay=1.0)
+@pytest.mark.parametrize("n", [5, 300])
+def test_step_host_matches_oracle(dl, mode, n):
+    from oracle import dlion_oracle as orc
+    w = inputs.custom([70000, 333] if n < 256 else [9000, 333], n, mode, "bf16", scale=1e-3, lr=1e-3, weight_decay=1.0)
     dev = torch.device("cuda:0")
     N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
     ctx = gp.make_ctx(dl, w)
@@ -158,8 +167,9 @@ def test_step_host_matches_oracle(dl, mode):
     x = x0.to(dev)
     packed = torch.zeros(N, W, dtype=torch.int32, device=dev)
     staging = torch.empty(2, D, dtype=torch.bfloat16, device=dev)
-    wire = torch.zeros(D if mode == AVG else W * 4, dtype=torch.uint8, device=dev)
-    host_wire = torch.zeros(wire.shape, dtype=torch.uint8).pin_memory()
+    K = ctx.delta_planes()
+    wire = torch.zeros(K * W, dtype=torch.int32, device=dev)
+    host_wire = torch.zeros(K * W, dtype=torch.int32).pin_memory()
     host_g = torch.empty(N, D, dtype=torch.bfloat16).pin_memory()
     for t in range(4):
         inputs.fill_grads(w, t, host_g)
@@ -169,8 +179,9 @@ def test_step_host_matches_oracle(dl, mode):
         gp.compare("packed", packed.cpu().numpy().view(np.uint32), ora.packed, True)
         gp.compare("m", m.cpu().numpy(), ora.m, False)
         gp.compare("x", x.cpu().numpy(), ora.x[mode], False)
-        want = ora.count[mode] if mode == AVG else ora.dbits[mode].view(np.uint8)
-        gp.compare("wire", host_wire.numpy(), want, True)
+        want = np.zeros(K * W, np.uint32)               # the broadcast message, from the oracle's own votes
+        orc.aggregate(w.segments, D, N, mode, ora.packed, want)
+        gp.compare("wire", host_wire.numpy().view(np.uint32), want, True)
     ctx.destroy()
 
 

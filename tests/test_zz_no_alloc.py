@@ -53,6 +53,47 @@ def test_sizes_beyond_the_fixed_scratch_are_rejected(dl):
         with pytest.raises(dl.DlionError) as e:
             dl.step_static(d, n, 0.9, 0.99, 1e-4, 0.0, 0, 0, t, t, t)
         assert e.value.status == dl.EINVAL
+    longer = torch.zeros(1028, device=dev)
     with pytest.raises(dl.DlionError) as e:
-        dl.step_static(1024, 1, 0.9, 0.99, 1e-4, 0.0, 0, 0, t[1:], t, t)
+        dl.step_static(1024, 1, 0.9, 0.99, 1e-4, 0.0, 0, 0, longer[1:], t, t)     # 4-byte aligned only
     assert e.value.status == dl.EALIGN
+    with pytest.raises(ValueError):                          # shorter than the call's extent: nothing is launched
+        dl.step_static(1024, 1, 0.9, 0.99, 1e-4, 0.0, 0, 0, t[1:], t, t)
+
+
+def test_against_the_oracle_big_then_small_and_nothing_allocated(dl):
+    """The entry point against the CPU oracle itself (not only against the regular CUDA path),
+    a large problem followed by a smaller one with another worker count on the same scratch
+    (the small one must not see the large one's stale sign bits), and the device's free memory
+    unchanged across the calls after the first one (which is the set-up call)."""
+    from oracle import dlion_oracle as orc
+    dev = torch.device("cuda:0")
+    warm = torch.zeros(128, device=dev)
+    dl.step_static(128, 1, 0.9, 0.99, 1e-4, 0.0, 0, 0, warm, warm.clone(), warm.clone())   # set-up call
+    torch.cuda.synchronize()
+    cases = [(2_000_003, 33, inputs.AVERAGE, "bf16"), (70_001, 5, inputs.MAJORITY, "f32"),
+             (4096 * 3 + 17, 300, inputs.AVERAGE, "f32")]
+    prepared = []
+    for d, n, mode, gd in cases:
+        w = inputs.custom([d], n, mode, gd, scale=1.0 if gd == "f32" else 1e-3, lr=1e-3, weight_decay=0.5)
+        gdt = inputs.grad_torch_dtype(w)
+        g = [inputs.fill_grads(w, t, torch.empty(n, w.d_pad, dtype=gdt)) for t in range(2)]
+        x0 = inputs.fill_x0(w, torch.empty(w.d_pad))
+        prepared.append((w, g, [t.to(dev) for t in g], x0, x0.to(dev), torch.zeros(n, w.d_pad, device=dev)))
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for w, g_cpu, g_dev, x0, x, m in prepared:
+        for t in range(2):
+            dl.step_static(w.d, w.n_workers, w.beta1, w.beta2, w.lr, w.weight_decay, w.mode, gp.gdtype_of(w),
+                           g_dev[t], m, x)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before       # six steps, not a byte taken from the device
+    for w, g_cpu, g_dev, x0, x, m in prepared:
+        n, D = w.n_workers, w.d_pad
+        m_ref, x_ref = np.zeros((n, D), np.float32), x0.numpy().copy()
+        for t in range(2):
+            packed = np.zeros((n, D // 32), np.uint32)
+            orc.worker_step(w.segments, D, n, inputs.as_numpy_grads(g_cpu[t]), m_ref, packed, w.beta1, w.beta2, nthreads=8)
+            orc.aggregate_apply(w.segments, D, n, w.mode, packed, x_ref, w.lr, w.weight_decay, nthreads=8)
+        assert gp.compare(f"d={w.d} N={n} m", m.cpu().numpy(), m_ref, False) == 0
+        assert gp.compare(f"d={w.d} N={n} x", x.cpu().numpy(), x_ref, False) == 0
