@@ -33,18 +33,27 @@ METRIC = "dlion_step_param_worker_updates_per_s"
 UNIT = "G param*worker updates/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes per launch of the worker-side kernel from an ncu capture
-# (dram__bytes_read.sum + dram__bytes_write.sum), as bytes per param*worker, keyed
-# by the SHA-256 of the kernel's source at capture time: reported only while the
-# source is unchanged.  See profiles/.
-NCU_TRAFFIC = {("worker_step_kernel", "e92caa95f78d0733"): 10.0759}   # profiles/worker_step_kernel_c2.md
+NCU_TRAFFIC_FILE = os.path.join(ROOT, "profiles", "ncu_traffic.json")
 
 
 def kernel_hash() -> str:
+    """SHA-256 (first 16 hex digits) of the worker-side kernel's sources."""
     h = hashlib.sha256()
     for name in ("worker_step.cu", "dlion_common.cuh"):
         h.update(open(os.path.join(ROOT, "paper_2404_00438_b200", "csrc", name), "rb").read())
     return h.hexdigest()[:16]
+
+
+def ncu_traffic(kernel: str, variant: str):
+    """DRAM bytes per param*worker of `kernel` from its ncu capture (dram__bytes_read.sum +
+    dram__bytes_write.sum over the units of the captured launch), as recorded in
+    profiles/ncu_traffic.json beside the hash of the kernel's sources at capture time; None
+    when there is no record or the sources have changed since."""
+    try:
+        rec = json.load(open(NCU_TRAFFIC_FILE))[kernel][variant]
+    except Exception:
+        return None
+    return float(rec["dram_bytes_per_param_worker"]) if rec.get("source_sha16") == kernel_hash() else None
 
 
 def measured_peak():
@@ -163,12 +172,12 @@ def mode_of(name: str) -> int:
     return {"majority": inputs.MAJORITY, "average": inputs.AVERAGE}[name]
 
 
-def oracle_sample_rate(w, mode: int, seconds: float, nthreads: int):
-    """Times the CPU oracle (as it stands) on a bounded sample: the first 2^22
+def oracle_sample_rate(w, mode: int, seconds: float, nthreads: int, n_max: int = 1 << 22):
+    """Times the CPU oracle (as it stands) on a bounded sample: the first n_max (2^22)
     arena coordinates of the workload, all N workers, repeated steps."""
     from oracle import dlion_oracle as orc
     orc.build()
-    n = min(w.d_pad, 1 << 22)
+    n = min(w.d_pad, n_max)
     segs = []
     for off, cnt in w.segments:
         a, b = off, min(off + cnt, n)
@@ -334,6 +343,37 @@ def run_ours(args):
     total_ms = ev[0][0].elapsed_time(ev[-1][2])
     clocks = sampler.stop() if rank == 0 else None
 
+    # ---- after the timed region: the server-side kernel under the OTHER aggregation rule
+    # (the workload names both), and the Global-Lion comparison step (the full-precision
+    # scheme the paper measures Distributed Lion against), K launches each on a scratch
+    # copy of x with events around every launch.  Neither enters `value`.
+    extra = {}
+    if args.path == "two_stage" and not args.no_extra:
+        other = inputs.AVERAGE if mode == inputs.MAJORITY else inputs.MAJORITY
+        x_scratch = x.clone()
+        ctx2 = dlion.Dlion(w.segments, D, N, w.beta1, w.beta2, w.lr, w.weight_decay, other,
+                           dlion.GRAD_F32 if w.grad_dtype == "f32" else dlion.GRAD_BF16)
+
+        def timed(fn):
+            for _ in range(3):
+                fn()
+            barrier()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+            e[0].record(stream)
+            for t in range(args.steps):
+                fn()
+                e[t + 1].record(stream)
+            barrier()
+            return statistics.mean(e[t].elapsed_time(e[t + 1]) for t in range(args.steps))
+
+        extra["other_rule_ms"] = timed(lambda: ctx2.aggregate_apply(packed, x_scratch))
+        extra["other_rule"] = "average" if other else "majority"
+        if args.state == "f32":
+            extra["global_lion_ms"] = timed(lambda: ctx2.step_global(g, m, x_scratch))
+        extra["launches"] = ctx2.launch_count()
+        ctx2.destroy()
+        del x_scratch
+
     # ---- optional: the same K steps captured once in a CUDA graph and replayed
     # (small workloads are bound by launch latency; the calls never synchronise)
     graph_ms = None
@@ -385,7 +425,7 @@ def run_ours(args):
             alg_bytes = w.d * N * bytes_per_param_worker_k1(w, sbytes)
             name = "worker_step_kernel"
         achieved = alg_bytes / (k1 * 1e-3) / 1e9
-        traffic = NCU_TRAFFIC.get((name, kernel_hash())) if sbytes == 4 and w.grad_dtype == "bf16" else None
+        traffic = ncu_traffic(name, f"grads_{w.grad_dtype}_momentum_{args.state}")
         roofline = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_source": peak_src, "frac_of_8tbs_nominal": achieved / 8000.0,
                     "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": k1,
@@ -395,14 +435,40 @@ def run_ours(args):
             b2 = w.d * bytes_per_param_k2(w)
             if args.path == "wire":                   # votes in, K planes out; K planes in, x in and out
                 b2 += 2 * w.d * ctx.delta_planes() / 8
-            stages = {("aggregate_kernel+apply_delta_kernel" if args.path == "wire" else "aggregate_apply_kernel"): {"achieved": b2 / (k2 * 1e-3) / 1e9, "unit": "GB/s",
-                                                 "frac": b2 / (k2 * 1e-3) / 1e9 / peak, "ms_per_launch": k2,
-                                                 "algorithmic_bytes_per_launch": b2}}
+            rule = "average" if mode else "majority"
+            key = ("aggregate_kernel+apply_delta_kernel<%s>" if args.path == "wire" else "aggregate_apply_kernel<%s>") % rule
+            stages = {key: {"achieved": b2 / (k2 * 1e-3) / 1e9, "unit": "GB/s",
+                            "frac": b2 / (k2 * 1e-3) / 1e9 / peak,
+                            "frac_of_8tbs_nominal": b2 / (k2 * 1e-3) / 1e9 / 8000.0, "ms_per_launch": k2,
+                            "algorithmic_bytes_per_launch": b2}}
+        comparison = None
+        if extra:
+            b2 = w.d * bytes_per_param_k2(w)
+            ms2 = extra["other_rule_ms"]
+            stages["aggregate_apply_kernel<%s>" % extra["other_rule"]] = {
+                "achieved": b2 / (ms2 * 1e-3) / 1e9, "unit": "GB/s", "frac": b2 / (ms2 * 1e-3) / 1e9 / peak,
+                "frac_of_8tbs_nominal": b2 / (ms2 * 1e-3) / 1e9 / 8000.0, "ms_per_launch": ms2,
+                "algorithmic_bytes_per_launch": b2,
+                "note": "timed after the timed region on a scratch copy of x; not part of `value`"}
+            if "global_lion_ms" in extra:
+                msg = extra["global_lion_ms"]
+                bg = w.d * (N * (w.grad_bytes + 8) + 8)
+                comparison = {"global_lion": {
+                    "call": "dlion_step_global (fp32 mean of the workers' blends, one sign; one launch)",
+                    "ms_per_step": msg, "value": w.d * N / (msg * 1e-3) / 1e9, "unit": UNIT,
+                    "achieved_gbs": bg / (msg * 1e-3) / 1e9, "algorithmic_bytes_per_launch": bg,
+                    "wire_bytes_each_way_per_worker": ctx.wire_bytes(2),
+                    "distributed_lion_ms_per_step": total_ms_max / args.steps,
+                    "note": "on one GPU both schemes read the same gradients and momenta, so their step "
+                            "times are close; the schemes differ in what crosses the network "
+                            "(wire_bytes_per_step)"}}
         cpu = None
         if not args.no_cpu_baseline and world == 1:
             cores = os.cpu_count() or 1
             rate, sample, _, _ = oracle_sample_rate(w, mode, args.cpu_seconds, cores)
-            cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+            rate1, sample1, _, _ = oracle_sample_rate(w, mode, args.cpu_seconds / 3, 1, n_max=1 << 20)
+            cpu = {"value": rate, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                   "single_thread": {"value": rate1, "unit": UNIT, "cores": 1, "sample": sample1}}
         up, down = ctx.wire_bytes(0), ctx.wire_bytes(1)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -416,7 +482,8 @@ def run_ours(args):
                        "timed_region": "K steps back to back in one bracket, on the last generated gradients",
                        "per_rank": "each rank steps its own full-size coordinate slab; no collective"},
             "ms_per_step_fresh_grads": fresh_ms, "ms_per_step_graph_replay": graph_ms,
-            "roofline": roofline, "roofline_stages": stages, "cpu_baseline": cpu, "e2e": e2e,
+            "roofline": roofline, "roofline_stages": stages, "comparison": comparison,
+            "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches, "clocks": clocks,
             "wire_bytes_per_step": {"up_all_workers": up, "down_per_worker": down,
                                     "fp32_gradients_each_way_per_worker": ctx.wire_bytes(2),
@@ -550,6 +617,8 @@ def main():
                     help="server: time the server-side kernel alone on the workload's wire buffer (1 GPU)")
     ap.add_argument("--graph", action="store_true", help="also time the K steps replayed from one CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the stages timed after the timed region (other aggregation rule, Global Lion)")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--e2e-warmup", type=int, default=1)
     ap.add_argument("--no-cpu-baseline", action="store_true")

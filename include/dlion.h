@@ -156,6 +156,19 @@ dlion_status dlion_aggregate(dlion_ctx* ctx, const uint32_t* packed, uint32_t* d
 dlion_status dlion_apply_delta(dlion_ctx* ctx, const uint32_t* delta_wire, float* x,
                                void* cuda_stream);
 
+/* dlion_apply_delta for a message assembled by an all-gather.  When the server's work
+ * is spread over S ranks (rank r votes on coordinate slice r and sends its part of the
+ * message to everyone -- the 1-bit analogue of reduce-scatter + all-gather of the
+ * exchange in Algorithm 1), the parts arrive slice after slice:
+ *   delta_wire  in  [S][K][slice_words]: for slice r, its K = dlion_delta_planes(ctx)
+ *               planes of slice_words words each (arena words r*slice_words ..), i.e.
+ *               word j of plane p of slice r at delta_wire[(r*K + p)*slice_words + j]
+ *   slice_words     words per slice; must divide d_pad/32 (DLION_EINVAL otherwise);
+ *                   0 means the plane-major layout of dlion_apply_delta
+ * Same update, same results; the parts are read where the collective put them. */
+dlion_status dlion_apply_delta_sliced(dlion_ctx* ctx, const uint32_t* delta_wire, uint64_t slice_words,
+                                      float* x, void* cuda_stream);
+
 /* Number of d-bit planes of the server->worker message: 1 for Majority Vote,
  * ceil(log2(N+1)) for Averaging (the paper's "log(N) bits" per parameter).
  * 0 for a null context. */

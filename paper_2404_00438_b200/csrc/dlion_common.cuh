@@ -70,6 +70,24 @@ __device__ __forceinline__ uint32_t lion_coord(float g, float& m, const Betas& k
     return c >= 0.0f ? 1u : 0u;
 }
 
+// The same for two coordinates at once with the packed binary32 instructions of
+// sm_100 (mul/add .rn.f32x2: each element rounded to nearest exactly like the
+// scalar form, so the results are the same bits; half the issue slots).  Returns
+// the two sign bits, coordinate 0 in bit 0.
+__device__ __forceinline__ uint32_t lion_pair(float2 g, float2& m, const Betas& k) {
+    const float2 c = __fadd2_rn(__fmul2_rn(make_float2(k.b1, k.b1), m), __fmul2_rn(make_float2(k.om1, k.om1), g));
+    m = __fadd2_rn(__fmul2_rn(make_float2(k.b2, k.b2), m), __fmul2_rn(make_float2(k.om2, k.om2), g));
+    return (c.x >= 0.0f ? 1u : 0u) | (c.y >= 0.0f ? 2u : 0u);
+}
+
+// Four consecutive coordinates held as float4: returns their sign nibble.
+__device__ __forceinline__ uint32_t lion_quad(const float4& g, float4& m, const Betas& k) {
+    float2 lo = make_float2(m.x, m.y), hi = make_float2(m.z, m.w);
+    const uint32_t nib = lion_pair(make_float2(g.x, g.y), lo, k) | (lion_pair(make_float2(g.z, g.w), hi, k) << 2);
+    m = make_float4(lo.x, lo.y, hi.x, hi.y);
+    return nib;
+}
+
 // Section 3.2, last equation: x - lr*(Delta + lambda*x).
 __device__ __forceinline__ float apply_coord(float x, float delta, float lr, float wd) {
     return __fsub_rn(x, __fmul_rn(lr, __fadd_rn(delta, __fmul_rn(wd, x))));
@@ -245,6 +263,7 @@ struct WireParams {                  // server-only aggregate / worker-side appl
     unsigned long long w_stride;     // words between consecutive binary vectors in packed
     unsigned long long plane_stride; // words between consecutive planes of the message
     uint32_t kplanes;                // planes in the message: 1, or ceil(log2(N+1)) for Averaging
+    unsigned long long slice_words;  // apply: 0, or the message is [slice][plane][slice_words] (all-gather order)
     float lr, wd;
     int average;
 };

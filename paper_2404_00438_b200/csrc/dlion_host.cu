@@ -132,7 +132,13 @@ dlion_status dlion_aggregate(dlion_ctx* ctx, const uint32_t* packed, uint32_t* d
 }
 
 dlion_status dlion_apply_delta(dlion_ctx* ctx, const uint32_t* delta_wire, float* x, void* cuda_stream) {
+    return dlion_apply_delta_sliced(ctx, delta_wire, 0, x, cuda_stream);
+}
+
+dlion_status dlion_apply_delta_sliced(dlion_ctx* ctx, const uint32_t* delta_wire, uint64_t slice_words,
+                                      float* x, void* cuda_stream) {
     if (ctx == nullptr || delta_wire == nullptr || x == nullptr) return DLION_EINVAL;
+    if (slice_words != 0 && (ctx->d_pad / 32) % slice_words != 0) return DLION_EINVAL;   // whole slices only
     if (!aligned16(delta_wire) || !aligned16(x)) return DLION_EALIGN;
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
@@ -145,7 +151,8 @@ dlion_status dlion_apply_delta(dlion_ctx* ctx, const uint32_t* delta_wire, float
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
     p.w_stride = ctx->d_pad / 32;
-    p.plane_stride = ctx->d_pad / 32;
+    p.plane_stride = slice_words != 0 ? slice_words : ctx->d_pad / 32;
+    p.slice_words = slice_words;
     p.kplanes = dlion_delta_planes(ctx);
     p.lr = ctx->lr;
     p.wd = ctx->wd;

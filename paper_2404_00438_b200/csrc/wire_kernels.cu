@@ -75,13 +75,20 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
 #pragma unroll
             for (int c = 0; c < 8; ++c) xv[c] = *(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
         }
+        // where my word of plane 0 sits: planes contiguous over all coordinates, or the
+        // all-gather order [slice][plane][slice_words] (plane_stride = slice_words then)
+        unsigned long long at = word_idx;
+        if (p.slice_words != 0) {
+            const unsigned long long r = word_idx / p.slice_words;
+            at = r * p.slice_words * p.kplanes + (word_idx - r * p.slice_words);
+        }
         uint32_t dword = 0;
         if constexpr (AVG) {
             uint32_t pl[kMaxPlanes];
 #pragma unroll
             for (int q = 0; q < kMaxPlanes; ++q) {
                 pl[q] = (q < PLANES && q < static_cast<int>(p.kplanes) && live)
-                            ? __ldg(p.wire_in + q * p.plane_stride + word_idx) : 0u;
+                            ? __ldg(p.wire_in + q * p.plane_stride + at) : 0u;
             }
             if (!have_table) {
                 fill_avg_table<PLANES>(avg_table, n, lane);
@@ -89,7 +96,7 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
             }
             publish_counts<PLANES>(pl, area, lane);
         } else {
-            dword = live ? __ldg(p.wire_in + word_idx) : 0u;
+            dword = live ? __ldg(p.wire_in + at) : 0u;
         }
 #pragma unroll
         for (int c = 0; c < 8; ++c) {

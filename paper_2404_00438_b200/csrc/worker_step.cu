@@ -44,26 +44,58 @@ worker_step_kernel(const WorkerParams p) {
 
         if (t.valid == kTile) {
             // ---- full tile: vector path, all loads issued before any use ----
-            const unsigned long long e0 = wbase + t.base + in_tile + lane * 4;
-            float4 g[kChunksPerWarp], m[kChunksPerWarp];
+            if constexpr (BF16 && MB16) {
+                // both streams are bf16: lane l of a 256-coordinate chunk holds coordinates
+                // 8l..8l+7 (one 16-byte access each for g and m), its eight signs are a byte,
+                // and four lanes' bytes make a word (two xor-shuffles)
+                const unsigned long long e0 = wbase + t.base + in_tile + lane * 8;
+                const uint16_t* gp = static_cast<const uint16_t*>(p.g) + e0;
+                uint16_t* mp = static_cast<uint16_t*>(p.m) + e0;
+                uint4 gv[2], mv[2];
 #pragma unroll
-            for (int u = 0; u < kChunksPerWarp; ++u) {
-                g[u] = load_grad4<BF16>(p.g, e0 + u * kChunk);
-                m[u] = load_state4<MB16>(p.m, e0 + u * kChunk);
-            }
-            uint32_t mine = 0;
+                for (int u = 0; u < 2; ++u) {
+                    gv[u] = *reinterpret_cast<const uint4*>(gp + u * 2 * kChunk);
+                    mv[u] = *reinterpret_cast<const uint4*>(mp + u * 2 * kChunk);
+                }
+                uint32_t mine = 0;
 #pragma unroll
-            for (int u = 0; u < kChunksPerWarp; ++u) {
-                uint32_t nib = lion_coord(g[u].x, m[u].x, k);
-                nib |= lion_coord(g[u].y, m[u].y, k) << 1;
-                nib |= lion_coord(g[u].z, m[u].z, k) << 2;
-                nib |= lion_coord(g[u].w, m[u].w, k) << 3;
-                store_state4<MB16>(p.m, e0 + u * kChunk, m[u]);
-                const uint32_t w = gather_word(nib, lane);
-                if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
+                for (int u = 0; u < 2; ++u) {
+                    const uint32_t gw[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
+                    const uint32_t mw[4] = {mv[u].x, mv[u].y, mv[u].z, mv[u].w};
+                    uint32_t out[4], byte = 0;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float2 m2 = make_float2(bf16_lo(mw[q]), bf16_hi(mw[q]));
+                        byte |= lion_pair(make_float2(bf16_lo(gw[q]), bf16_hi(gw[q])), m2, k) << (2 * q);
+                        out[q] = pack_bf16x2_rne(m2.x, m2.y);
+                    }
+                    *reinterpret_cast<uint4*>(mp + u * 2 * kChunk) = make_uint4(out[0], out[1], out[2], out[3]);
+                    uint32_t w = byte << (8u * (lane & 3u));
+                    w |= __shfl_xor_sync(kFull, w, 1);
+                    w |= __shfl_xor_sync(kFull, w, 2);
+                    if ((lane & 3u) == static_cast<uint32_t>(u)) mine = w;
+                }
+                // lane l (l%4 < 2) holds word l/4 of chunk l%4: word index 8*(l%4) + l/4
+                if ((lane & 3u) < 2u) words[8u * (lane & 3u) + (lane >> 2)] = mine;
+            } else {
+                const unsigned long long e0 = wbase + t.base + in_tile + lane * 4;
+                float4 g[kChunksPerWarp], m[kChunksPerWarp];
+#pragma unroll
+                for (int u = 0; u < kChunksPerWarp; ++u) {
+                    g[u] = load_grad4<BF16>(p.g, e0 + u * kChunk);
+                    m[u] = load_state4<MB16>(p.m, e0 + u * kChunk);
+                }
+                uint32_t mine = 0;
+#pragma unroll
+                for (int u = 0; u < kChunksPerWarp; ++u) {
+                    const uint32_t nib = lion_quad(g[u], m[u], k);
+                    store_state4<MB16>(p.m, e0 + u * kChunk, m[u]);
+                    const uint32_t w = gather_word(nib, lane);
+                    if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
+                }
+                // lane l (l%8 < 4) holds the word of chunk l%8, group l/8: word index 4*(l%8) + l/8
+                if ((lane & 7u) < kChunksPerWarp) words[4u * (lane & 7u) + (lane >> 3)] = mine;
             }
-            // lane l (l%8 < 4) holds the word of chunk l%8, group l/8: word index 4*(l%8) + l/8
-            if ((lane & 7u) < kChunksPerWarp) words[4u * (lane & 7u) + (lane >> 3)] = mine;
         } else {
             // ---- last tile of a segment: per-coordinate guards -------------
 #pragma unroll 1

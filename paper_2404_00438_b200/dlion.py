@@ -24,7 +24,8 @@ OK, EINVAL, EALIGN, ENOMEM, ECUDA, ESTATE = range(6)
 
 EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_set_momentum_dtype",
            "dlion_set_worker_betas", "dlion_worker_step",
-           "dlion_aggregate_apply", "dlion_aggregate", "dlion_apply_delta", "dlion_delta_planes",
+           "dlion_aggregate_apply", "dlion_aggregate", "dlion_apply_delta", "dlion_apply_delta_sliced",
+           "dlion_delta_planes",
            "dlion_step_fused", "dlion_step_global", "dlion_step_host", "dlion_step_static",
            "dlion_wire_bytes",
            "dlion_launch_count", "dlion_status_str", "dlion_destroy")
@@ -67,6 +68,8 @@ def _load() -> ctypes.CDLL:
     lib.dlion_aggregate.restype = i32
     lib.dlion_apply_delta.argtypes = [vp, vp, vp, vp]
     lib.dlion_apply_delta.restype = i32
+    lib.dlion_apply_delta_sliced.argtypes = [vp, vp, u64, vp, vp]
+    lib.dlion_apply_delta_sliced.restype = i32
     lib.dlion_delta_planes.argtypes = [vp]
     lib.dlion_delta_planes.restype = u32
     lib.dlion_step_fused.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -241,6 +244,12 @@ class Dlion:
         self._t(x, "x", (torch.float32,), self.d_pad)
         self._check(_lib.dlion_apply_delta(self._ctx, _ptr(delta_wire), _ptr(x), _stream()),
                     "dlion_apply_delta")
+
+    def apply_delta_sliced(self, delta_wire: torch.Tensor, slice_words: int, x: torch.Tensor) -> None:
+        self._t(delta_wire, "delta_wire", _WORD_DTYPES, self.delta_planes() * self.words)
+        self._t(x, "x", (torch.float32,), self.d_pad)
+        self._check(_lib.dlion_apply_delta_sliced(self._ctx, _ptr(delta_wire), int(slice_words), _ptr(x),
+                                                  _stream()), "dlion_apply_delta_sliced")
 
     def delta_planes(self) -> int:
         return int(_lib.dlion_delta_planes(self._ctx))

@@ -9,7 +9,8 @@ spread over the workers, the 1-bit analogue of reduce-scatter + all-gather:
   2. all-to-all of bit shards       rank r receives coordinate slice r of every worker
   3. vote on the slice, local       the broadcast message for slice r (1 or K bit planes)
   4. all-gather of the message      every rank now holds Delta for all d coordinates
-  5. apply, local                   x <- x - eps (Delta + lambda x)
+  5. apply, local                   x <- x - eps (Delta + lambda x), the message read
+                                    slice by slice where the all-gather put it
 
 Per rank and step this moves d*(world-1)/world/8 bytes out in step 2 and
 K*d*(world-1)/world/8 bytes in step 4 (K = 1 for Majority Vote,
@@ -17,7 +18,7 @@ ceil(log2(N+1)) for Averaging): Table 1 of the paper, against 4d bytes each way
 for an fp32 gradient exchange.
 
 Steps 1, 3 and 5 are three calls of the C ABI (``dlion_worker_step``,
-``dlion_aggregate``, ``dlion_apply_delta``); steps 2 and 4 are
+``dlion_aggregate``, ``dlion_apply_delta_sliced``); steps 2 and 4 are
 ``torch.distributed`` collectives (NCCL on GPUs).  Received shards land in this
 rank's own memory and are read with ordinary loads.  This module only
 orchestrates; it holds no optimizer arithmetic.  The three local steps are
@@ -40,47 +41,51 @@ def padded_length(d_pad: int, world: int) -> int:
     return (d_pad + q - 1) // q * q
 
 
-def planes(n_workers: int, mode: int) -> int:
-    """Bit planes of the broadcast message: 1 (Majority Vote) or ceil(log2(N+1)) (Averaging)."""
-    return 1 if mode == 0 else max(1, n_workers.bit_length())
-
-
 class DlionKernels:
-    """The three local steps on this rank's GPU through the CUDA library."""
+    """The three local steps on this rank's GPU through the CUDA library.
+
+    Two contexts: one over the model's segment table with N = world workers (this rank steps
+    worker ``rank`` of it, and applies the broadcast update), and a flat one over this rank's
+    coordinate slice (the vote on the slice: padding between tensors is voted on too, which
+    is harmless because the apply never touches padding)."""
 
     def __init__(self, segments, d_pad_x: int, world: int, rank: int, beta1: float, beta2: float,
                  lr: float, weight_decay: float, mode: int, gdtype: int):
         from . import dlion
+        self.rank = rank
         slice_len = d_pad_x // world
-        # this rank as a worker: one worker's state over the whole model
-        self.worker = dlion.Dlion(segments, d_pad_x, 1, beta1, beta2, lr, weight_decay, mode, gdtype)
-        # this rank as the server of its slice: all workers' bits for slice_len coordinates
+        self.model = dlion.Dlion(segments, d_pad_x, world, beta1, beta2, lr, weight_decay, mode, gdtype)
         self.server = dlion.Dlion([(0, slice_len)], slice_len, world, beta1, beta2, lr, weight_decay,
                                   mode, gdtype)
-        # every rank applies the broadcast update to its copy of x
-        self.applier = dlion.Dlion(segments, d_pad_x, world, beta1, beta2, lr, weight_decay, mode, gdtype)
+
+    def delta_planes(self) -> int:
+        return self.model.delta_planes()
 
     def set_lr(self, lr: float) -> None:
-        self.applier.set_lr(lr)
+        self.model.set_lr(lr)
 
     def worker_step(self, g: torch.Tensor, m: torch.Tensor, packed: torch.Tensor) -> None:
-        self.worker.worker_step(0, g, m, packed)
+        self.model.worker_step(self.rank, g, m, packed)
 
     def aggregate(self, packed_slices: torch.Tensor, wire_slice: torch.Tensor) -> None:
         self.server.aggregate(packed_slices, wire_slice)
 
-    def apply_delta(self, wire: torch.Tensor, x: torch.Tensor) -> None:
-        self.applier.apply_delta(wire, x)
+    def apply_delta_sliced(self, gathered: torch.Tensor, slice_words: int, x: torch.Tensor) -> None:
+        self.model.apply_delta_sliced(gathered, slice_words, x)
 
 
 class DistributedLion:
     """One rank of Distributed Lion.  ``g``, ``m``, ``x`` have ``d_pad_x`` elements
-    (``padded_length(d_pad, world)``); ``m`` is this worker's own momentum."""
+    (``padded_length(d_pad, world)``); ``m`` is this worker's own momentum.
+
+    ``host_staged = True`` routes the two collectives through pinned host buffers (for
+    process groups that only move host memory, such as gloo); the default hands the device
+    buffers to the group's backend (NCCL)."""
 
     def __init__(self, segments: Sequence[Tuple[int, int]], d_pad: int, mode: int, kernels=None,
                  beta1: float = 0.9, beta2: float = 0.99, lr: float = 1e-4, weight_decay: float = 0.0,
                  gdtype: int = 0, group: Optional[dist.ProcessGroup] = None,
-                 device: Optional[torch.device] = None):
+                 device: Optional[torch.device] = None, host_staged: bool = False):
         self.group = group
         self.world = dist.get_world_size(group)
         self.rank = dist.get_rank(group)
@@ -88,30 +93,50 @@ class DistributedLion:
         self.d_pad_x = padded_length(d_pad, self.world)
         self.words = self.d_pad_x // 32
         self.slice_words = self.words // self.world
-        self.k = planes(self.world, mode)
         self.kernels = kernels if kernels is not None else DlionKernels(
             segments, self.d_pad_x, self.world, self.rank, beta1, beta2, lr, weight_decay, mode, gdtype)
+        self.k = int(self.kernels.delta_planes())       # planes of the broadcast message, from the library
         dev = device if device is not None else torch.device("cuda", torch.cuda.current_device())
         z = dict(dtype=torch.int32, device=dev)
         self.packed = torch.zeros(self.words, **z)                           # my delta, all coordinates
         self.recv = torch.zeros(self.world, self.slice_words, **z)           # everyone's delta, my slice
         self.wire_slice = torch.zeros(self.k, self.slice_words, **z)         # message for my slice
+        # every slice's message, in the order the all-gather delivers them: [slice][plane][word]
         self.gathered = torch.zeros(self.world, self.k, self.slice_words, **z)
-        self.wire = torch.zeros(self.k, self.words, **z)                     # message, all coordinates
+        self.host_staged = bool(host_staged) and dev.type == "cuda"
+        if self.host_staged:
+            h = dict(dtype=torch.int32, pin_memory=True)
+            self.h_packed, self.h_recv = torch.zeros(self.words, **h), torch.zeros(self.words, **h)
+            self.h_slice = torch.zeros(self.k * self.slice_words, **h)
+            self.h_gathered = torch.zeros(self.world * self.k * self.slice_words, **h)
 
     def wire_bytes_per_step(self) -> Tuple[int, int]:
         """(bytes this rank sends in the all-to-all, bytes it receives in the all-gather)."""
         others = self.world - 1
         return others * self.slice_words * 4, others * self.k * self.slice_words * 4
 
+    def _all_to_all(self) -> None:
+        if not self.host_staged:
+            dist.all_to_all_single(self.recv.view(-1), self.packed, group=self.group)
+            return
+        self.h_packed.copy_(self.packed)                 # ordered on the current stream, then waits
+        dist.all_to_all_single(self.h_recv, self.h_packed, group=self.group)
+        self.recv.view(-1).copy_(self.h_recv, non_blocking=True)
+
+    def _all_gather(self) -> None:
+        if not self.host_staged:
+            dist.all_gather_into_tensor(self.gathered.view(-1), self.wire_slice.view(-1), group=self.group)
+            return
+        self.h_slice.copy_(self.wire_slice.view(-1))
+        dist.all_gather_into_tensor(self.h_gathered, self.h_slice, group=self.group)
+        self.gathered.view(-1).copy_(self.h_gathered, non_blocking=True)
+
     def step(self, g: torch.Tensor, m: torch.Tensor, x: torch.Tensor) -> None:
         self.kernels.worker_step(g, m, self.packed)
-        dist.all_to_all_single(self.recv.view(-1), self.packed, group=self.group)
+        self._all_to_all()
         self.kernels.aggregate(self.recv, self.wire_slice)
-        dist.all_gather_into_tensor(self.gathered.view(-1), self.wire_slice.view(-1), group=self.group)
-        # [rank][plane][slice word] -> [plane][rank][slice word] = plane-major over all coordinates
-        self.wire.view(self.k, self.world, self.slice_words).copy_(self.gathered.permute(1, 0, 2))
-        self.kernels.apply_delta(self.wire, x)
+        self._all_gather()
+        self.kernels.apply_delta_sliced(self.gathered, self.slice_words, x)   # read where the all-gather put them
 
 
 class LionOptimizer:

@@ -146,60 +146,259 @@ def run_small(dl, w: inputs.Workload, steps: int, path: str = "two_stage",
     return worst
 
 
-def pick_slabs(w: inputs.Workload, n_random: int = 3, width: int = 1 << 14, seed: int = 7):
-    """Arena ranges to check at full size: both ends, a few segment joints, random interiors."""
+# --------------------------------------------------------------------------
+# full-size runs: the oracle works slab by slab (coordinates are independent, so a
+# slab is a complete problem); what it produces is uploaded and compared on the GPU
+# --------------------------------------------------------------------------
+def ulp_diff_dev(a: torch.Tensor, b: torch.Tensor) -> int:
+    """ulp_diff for two float32 tensors on the same device (bounded temporaries)."""
+    assert a.dtype == torch.float32 and b.dtype == torch.float32 and a.shape == b.shape
+    ia, ib = a.reshape(-1).view(torch.int32), b.reshape(-1).view(torch.int32)
+    if torch.equal(ia, ib):
+        return 0
+    worst = 0
+    for c0 in range(0, ia.numel(), 1 << 26):
+        fa, fb = a.reshape(-1)[c0:c0 + (1 << 26)], b.reshape(-1)[c0:c0 + (1 << 26)]
+        nan_a, nan_b = torch.isnan(fa), torch.isnan(fb)
+        assert torch.equal(nan_a, nan_b), "NaN pattern differs"
+        ka, kb = (v.view(torch.int32).to(torch.int64) for v in (fa, fb))
+        ka = torch.where(ka < 0, -(ka & 0x7FFFFFFF), ka)
+        kb = torch.where(kb < 0, -(kb & 0x7FFFFFFF), kb)
+        d = (ka - kb).abs()
+        d[nan_a] = 0
+        worst = max(worst, int(d.max().item()))
+    return worst
+
+
+def bf16_ulp_diff_dev(a: torch.Tensor, b: torch.Tensor) -> int:
+    """Largest distance in bf16 units in the last place between two int16 tensors of bf16 bits."""
+    if a.numel() == 0 or torch.equal(a, b):
+        return 0
+    ka, kb = a.to(torch.int32), b.to(torch.int32)
+    ka = torch.where(ka < 0, -(ka & 0x7FFF), ka)
+    kb = torch.where(kb < 0, -(kb & 0x7FFF), kb)
+    return int((ka - kb).abs().max().item())
+
+
+def compare_dev(tag: str, got: torch.Tensor, want: torch.Tensor, exact: bool) -> int:
+    """got: the CUDA library's result (device); want: the oracle's, uploaded.  Integer and
+    byte data are compared bit for bit, float32 state within TOL_ULP."""
+    assert got.shape == want.shape and got.dtype == want.dtype, f"{tag}: shape or dtype differs"
+    if exact:
+        if not torch.equal(got, want):
+            bad = torch.nonzero(got.reshape(-1) != want.reshape(-1))
+            k = int(bad[0].item())
+            raise AssertionError(f"{tag}: {bad.numel()} mismatches, first at flat index {k}: "
+                                 f"got {got.reshape(-1)[k].item()!r} want {want.reshape(-1)[k].item()!r}")
+        return 0
+    u = ulp_diff_dev(got, want)
+    assert u <= TOL_ULP, f"{tag}: {u} ulp > {TOL_ULP}"
+    return u
+
+
+def _pinned(shape, dtype) -> torch.Tensor:
+    return torch.zeros(shape, dtype=dtype, pin_memory=True)
+
+
+class SlabOracle:
+    """The oracle's state of one arena range [lo, hi), in pinned host memory so that the
+    per-step uploads run at PCIe speed.  state = "bf16" keeps the momentum as bf16 bits."""
+
+    def __init__(self, w: inputs.Workload, lo: int, hi: int, modes: Sequence[int], state: str = "f32",
+                 counts: bool = True):
+        self.w, self.lo, self.hi, self.n, self.state = w, lo, hi, hi - lo, state
+        self.segs = clip_segments(w.segments, lo, hi)
+        N, n = w.n_workers, self.n
+        self.m = _pinned((N, n), torch.float32 if state == "f32" else torch.int16)
+        self.packed = _pinned((N, n // 32), torch.int32)
+        self.x = {md: _pinned((n,), torch.float32) for md in modes}
+        self.dbits = {md: _pinned((n // 32,), torch.int32) for md in modes}
+        self.count = {md: (_pinned((n,), torch.uint8) if counts and N <= 255 else None) for md in modes}
+
+    def reset(self, x0: torch.Tensor) -> None:
+        self.m.zero_()
+        for md in self.x:
+            self.x[md].copy_(x0)
+
+    def step(self, g: np.ndarray, nthreads: int) -> None:
+        w = self.w
+        m = self.m.numpy() if self.state == "f32" else self.m.numpy().view(np.uint16)
+        packed = self.packed.numpy().view(np.uint32)
+        if self.state == "f32":
+            orc.worker_step(self.segs, self.n, w.n_workers, g, m, packed, w.beta1, w.beta2, nthreads=nthreads)
+        else:
+            orc.worker_step_ex(self.segs, self.n, w.n_workers, g, m, packed, [w.beta1] * w.n_workers,
+                               [w.beta2] * w.n_workers, nthreads=nthreads)
+        for md in self.x:
+            orc.aggregate_apply(self.segs, self.n, w.n_workers, md, packed, self.x[md].numpy(), w.lr,
+                                w.weight_decay, delta_bits=self.dbits[md].numpy().view(np.uint32),
+                                count=None if self.count[md] is None else self.count[md].numpy(),
+                                nthreads=nthreads)
+
+
+def partition(d_pad: int, width: int):
+    """[0, d_pad) cut into consecutive ranges of at most `width` coordinates (a multiple of 128)."""
+    assert width % 128 == 0
+    return [(lo, min(lo + width, d_pad)) for lo in range(0, d_pad, width)]
+
+
+def pick_slabs(w: inputs.Workload, frac: float = 0.0, n_random: int = 3, width: int = 1 << 14,
+               interior: int = 1 << 20, seed: int = 7):
+    """Arena ranges to follow over many steps at full size: both ends, EVERY joint between two
+    tensors (a window of `width` coordinates around it), and random interior ranges -- n_random
+    of them, or as many ranges of `interior` coordinates as it takes to cover `frac` of the
+    arena.  Overlapping ranges are merged."""
     D = w.d_pad
     width = min(width, D)
-    slabs = {(0, width), (D - width, D)}
-    joints = [off for off, _ in w.segments[1:]]
+    want = [(0, width), (D - width, D)]
+    for off, _ in w.segments[1:]:
+        lo = max(0, min(D - width, (off - width // 2) // 128 * 128))
+        want.append((lo, lo + width))
     rng = np.random.default_rng(seed)
-    for j in ([joints[0], joints[len(joints) // 2], joints[-1]] if joints else []):
-        lo = max(0, min(D - width, (j - width // 2) // 128 * 128))
-        slabs.add((lo, lo + width))
-    for _ in range(n_random):
-        lo = int(rng.integers(0, max(1, (D - width) // 128))) * 128
-        slabs.add((lo, lo + width))
-    return sorted(slabs)
+    if frac > 0:
+        interior = min(interior, D)
+        for _ in range(int(np.ceil(frac * D / interior))):
+            lo = int(rng.integers(0, max(1, (D - interior) // 128 + 1))) * 128
+            want.append((lo, lo + interior))
+    else:
+        for _ in range(n_random):
+            lo = int(rng.integers(0, max(1, (D - width) // 128))) * 128
+            want.append((lo, lo + width))
+    merged = []
+    for lo, hi in sorted(want):
+        if merged and lo <= merged[-1][1]:
+            merged[-1] = (merged[-1][0], max(merged[-1][1], hi))
+        else:
+            merged.append((lo, hi))
+    return merged
 
 
 def run_full(dl, w: inputs.Workload, steps: int, path: str = "two_stage",
-             modes: Sequence[int] = (0, 1), slabs=None) -> int:
-    """Full-size run in the launch configuration the benchmark times; the oracle
-    recomputes sampled coordinate slabs from the same gradient bytes."""
+             modes: Sequence[int] = (0, 1), slabs=None, persist: bool = True, state: str = "f32",
+             width: int = 1 << 22) -> int:
+    """Full-size run in the launch configuration the benchmark times, checked against the
+    oracle on the arena ranges `slabs` (default: the whole arena, cut into ranges of `width`
+    coordinates) after EVERY step: packed signs, Delta bits and vote counts bit for bit,
+    momentum and parameters within TOL_ULP.  The oracle is fed the gradient bytes the
+    kernels read (copied out of the device arena).
+
+    persist = True keeps the oracle's state of every range on the host from step to step
+    (N * 4 bytes per covered coordinate).  persist = False holds one range at a time: after
+    step t the oracle replays steps 0..t of the range from m = 0 and x_0, the earlier steps'
+    gradients regenerated from the seed -- for arenas whose momentum does not fit host
+    memory.  Returns the largest ulp distance seen.
+    """
+    import os
     dev = torch.device("cuda:0")
     N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
     gdt = inputs.grad_torch_dtype(w)
-    slabs = slabs or pick_slabs(w)
+    nthreads = os.cpu_count() or 1
+    slabs = partition(D, width) if slabs is None else slabs
+    widest = max(hi - lo for lo, hi in slabs)
+    fused = path == "fused"
+    if fused:
+        assert len(modes) == 1
+    sdt = torch.float32 if state == "f32" else torch.bfloat16
     g = torch.empty(N, D, dtype=gdt, device=dev)
-    m = torch.zeros(N, D, device=dev)
+    m = torch.zeros(N, D, dtype=sdt, device=dev)
     x0 = inputs.fill_x0(w, torch.empty(D, device=dev))
     xs = {md: x0.clone() for md in modes}
-    del x0
+    if persist:
+        x0 = None
     packed = torch.zeros(N, W, dtype=torch.int32, device=dev)
+    dbits = {md: None if fused else torch.zeros(W, dtype=torch.int32, device=dev) for md in modes}
+    count = {md: (torch.zeros(D, dtype=torch.uint8, device=dev) if not fused and N <= 255 else None)
+             for md in modes}
     ctx = {md: make_ctx(dl, w, md) for md in modes}
-    oras = [OracleState(w, lo, hi, np.zeros((N, hi - lo), np.float32),
-                        xs[modes[0]][lo:hi].cpu().numpy(), modes) for lo, hi in slabs]
+    if state == "bf16":
+        for c in ctx.values():
+            c.set_momentum_dtype(dl.STATE_BF16)
+    g_stage = _pinned((N * widest,), torch.int16 if gdt == torch.bfloat16 else torch.float32)
+    if persist:
+        oras = [SlabOracle(w, lo, hi, modes, state, counts=not fused) for lo, hi in slabs]
+        for o in oras:
+            o.reset(xs[modes[0]][o.lo:o.hi])
+    else:
+        one = {}                                    # one oracle state per distinct range length
+        g_tmp = torch.empty(N, widest, dtype=gdt, device=dev)
+
+    def stage_grads(src: torch.Tensor, n: int) -> np.ndarray:
+        dst = g_stage[:N * n].view(N, n)
+        dst.copy_(src.view(torch.int16) if gdt == torch.bfloat16 else src)
+        a = dst.numpy()
+        return a.view(np.uint16) if gdt == torch.bfloat16 else a
+
     worst = 0
     for t in range(steps):
         inputs.fill_grads(w, t, g)
-        for o in oras:
-            o.step(inputs.as_numpy_grads(g[:, o.lo:o.hi]))
-        if path == "fused":
-            assert len(modes) == 1
+        if fused:
             ctx[modes[0]].step_fused(g, m, xs[modes[0]], packed)
         else:
             ctx[modes[0]].worker_step(-1, g, m, packed)
             for md in modes:
-                ctx[md].aggregate_apply(packed, xs[md])
+                ctx[md].aggregate_apply(packed, xs[md], dbits[md], count[md])
         torch.cuda.synchronize()
-        for o in oras:
-            tag = f"{w.name} N={N} step {t} slab [{o.lo},{o.hi}) {path}"
-            compare(tag + " packed", packed[:, o.lo // 32:o.hi // 32].cpu().numpy().view(np.uint32),
-                    o.packed, True)
-            worst = max(worst, compare(tag + " m", m[:, o.lo:o.hi].cpu().numpy(), o.m, False))
+        for k, (lo, hi) in enumerate(slabs):
+            n = hi - lo
+            if persist:
+                o = oras[k]
+                o.step(stage_grads(g[:, lo:hi], n), nthreads)
+            else:
+                if n not in one:
+                    one[n] = SlabOracle(w, 0, n, modes, state, counts=not fused)
+                o = one[n]
+                o.lo, o.hi, o.segs = lo, hi, clip_segments(w.segments, lo, hi)
+                o.reset(x0[lo:hi])
+                for s in range(t):
+                    o.step(stage_grads(inputs.fill_grads(w, s, g_tmp[:, :n], lo, hi), n), nthreads)
+                o.step(stage_grads(g[:, lo:hi], n), nthreads)
+            tag = f"{w.name} N={N} step {t} range [{lo},{hi}) {path} {state}"
+            compare_dev(tag + " packed", packed[:, lo // 32:hi // 32], o.packed.to(dev), True)
+            if state == "f32":
+                worst = max(worst, compare_dev(tag + " m", m[:, lo:hi], o.m.to(dev), False))
+            else:                                  # bf16 state: the tolerance is one bf16 ulp
+                u = bf16_ulp_diff_dev(m[:, lo:hi].view(torch.int16), o.m.to(dev))
+                assert u <= 1, f"{tag} m: {u} bf16 ulp"
+                worst = max(worst, u)
             for md in modes:
-                worst = max(worst, compare(tag + f" x mode {md}", xs[md][o.lo:o.hi].cpu().numpy(),
-                                           o.x[md], False))
+                worst = max(worst, compare_dev(tag + f" x mode {md}", xs[md][lo:hi], o.x[md].to(dev), False))
+                if not fused:
+                    compare_dev(tag + f" delta_bits mode {md}", dbits[md][lo // 32:hi // 32], o.dbits[md].to(dev), True)
+                    if count[md] is not None:
+                        compare_dev(tag + f" count mode {md}", count[md][lo:hi], o.count[md].to(dev), True)
     for c in ctx.values():
         c.destroy()
     return worst
+
+
+def cross_check_paths(dl, w: inputs.Workload, steps: int, mode: int) -> None:
+    """Whole arenas, no CPU work: the product paths that promise identical bits -- the
+    two-stage step, per-worker calls followed by dlion_aggregate + dlion_apply_delta, and the
+    one-launch step -- are run side by side on the same gradients and must leave identical
+    momentum, parameters and sign words everywhere, padding included.  (The oracle anchors the
+    two-stage path; this extends that anchor to every coordinate of the other paths.)"""
+    dev = torch.device("cuda:0")
+    N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
+    gdt = inputs.grad_torch_dtype(w)
+    ctx = make_ctx(dl, w, mode)
+    g = torch.empty(N, D, dtype=gdt, device=dev)
+    x0 = inputs.fill_x0(w, torch.empty(D, device=dev))
+    ms = [torch.zeros(N, D, device=dev) for _ in range(3)]
+    xs = [x0.clone() for _ in range(3)]
+    ps = [torch.zeros(N, W, dtype=torch.int32, device=dev) for _ in range(3)]
+    wire = torch.zeros(ctx.delta_planes() * W, dtype=torch.int32, device=dev)
+    for t in range(steps):
+        inputs.fill_grads(w, t, g)
+        ctx.worker_step(-1, g, ms[0], ps[0])
+        ctx.aggregate_apply(ps[0], xs[0])
+        for i in range(N):
+            ctx.worker_step(i, g[i], ms[1][i], ps[1][i])
+        ctx.aggregate(ps[1], wire)
+        ctx.apply_delta(wire, xs[1])
+        ctx.step_fused(g, ms[2], xs[2], ps[2])
+        torch.cuda.synchronize()
+        for k, name in ((1, "per-worker + wire"), (2, "fused")):
+            assert torch.equal(ms[k], ms[0]), f"{w.name} step {t}: momentum of the {name} path differs"
+            assert torch.equal(xs[k], xs[0]), f"{w.name} step {t}: parameters of the {name} path differ"
+            assert torch.equal(ps[k], ps[0]), f"{w.name} step {t}: sign words of the {name} path differ"
+    ctx.destroy()

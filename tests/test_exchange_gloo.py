@@ -41,9 +41,13 @@ class OracleKernels:
                            np.ascontiguousarray(packed_slices.numpy().view(np.uint32)), wire)
         wire_slice.copy_(torch.from_numpy(wire.view(np.int32)).view(k, -1))
 
-    def apply_delta(self, wire, x):
-        self.orc.apply_delta(self.segments, self.d, self.world, self.mode,
-                             np.ascontiguousarray(wire.numpy().view(np.uint32)).reshape(-1), x.numpy(),
+    def delta_planes(self):
+        return self.orc.delta_planes(self.world, self.mode)
+
+    def apply_delta_sliced(self, gathered, slice_words, x):
+        # [slice][plane][word] -> the plane-major message of the oracle's apply
+        wire = np.ascontiguousarray(gathered.numpy().view(np.uint32).transpose(1, 0, 2)).reshape(-1)
+        self.orc.apply_delta(self.segments, self.d, self.world, self.mode, wire, x.numpy(),
                              self.w.lr, self.w.weight_decay)
 
 

@@ -422,6 +422,58 @@ def test_more_than_255_workers(dl, n, mode):
     ctx.destroy()
 
 
+@pytest.mark.parametrize("n", [8191, 8192, 16383, 16384, 32768, 65535])
+@pytest.mark.parametrize("mode", [MAJ, AVG])
+def test_thirteen_to_sixteen_bit_planes(dl, n, mode):
+    """The largest worker counts the library accepts (13 to 16 bit planes of votes, 65535 =
+    DLION_MAX_WORKERS): the one-call server step, the server-only vote and the worker-side
+    apply against the oracle on a ragged table.  The sign words are drawn directly (the vote
+    does not care where they came from) with a different probability of +1 per coordinate, and
+    a few coordinates are forced to the extremes: all +1, all -1, an exact tie (even N) and one
+    vote short of it."""
+    from oracle import dlion_oracle as orc
+    w = inputs.custom([4096 + 77, 33, 1000], n, mode, "f32", lr=1e-2, weight_decay=0.5)
+    dev = torch.device("cuda:0")
+    D, W = w.d_pad, w.d_pad // 32
+    rng = np.random.default_rng(n + mode)
+    valid = np.zeros(D, bool)
+    for off, cnt in w.segments:
+        valid[off:off + cnt] = True
+    bits = rng.integers(0, 256, (n, D), dtype=np.uint8) < rng.integers(0, 257, D)[None, :]
+    half = (n + 1) // 2                                  # smallest count with Delta = +1
+    for seg_off in (w.segments[0][0], w.segments[2][0]):
+        bits[:, seg_off + 0] = True
+        bits[:, seg_off + 1] = False
+        bits[:, seg_off + 2] = np.arange(n) < half
+        bits[:, seg_off + 3] = np.arange(n) < half - 1
+        bits[:, seg_off + 4] = np.arange(n) >= n - half   # the same count held by the LAST workers
+    bits &= valid[None, :]
+    packed_np = np.packbits(bits, axis=1, bitorder="little").view(np.uint32).reshape(n, -1).copy()
+    x0 = inputs.fill_x0(w, torch.empty(D))
+    ctx = gp.make_ctx(dl, w)
+    K = ctx.delta_planes()
+    assert K == orc.delta_planes(n, mode) == (1 if mode == MAJ else int(n).bit_length())
+    wire_ref = np.zeros(K * W, np.uint32)
+    orc.aggregate(w.segments, D, n, mode, packed_np, wire_ref)
+    x_ref = x0.numpy().copy()
+    orc.apply_delta(w.segments, D, n, mode, wire_ref, x_ref, w.lr, w.weight_decay)
+    x_ref1, dbits_ref = x0.numpy().copy(), np.zeros(W, np.uint32)
+    orc.aggregate_apply(w.segments, D, n, mode, packed_np, x_ref1, w.lr, w.weight_decay, delta_bits=dbits_ref)
+    packed = torch.from_numpy(packed_np.view(np.int32)).to(dev)
+    wire = torch.zeros(K * W, dtype=torch.int32, device=dev)
+    dbits = torch.zeros(W, dtype=torch.int32, device=dev)
+    x, x_one = x0.to(dev), x0.to(dev)
+    ctx.aggregate(packed, wire)
+    ctx.apply_delta(wire, x)
+    ctx.aggregate_apply(packed, x_one, dbits)
+    torch.cuda.synchronize()
+    gp.compare("delta wire", wire.cpu().numpy().view(np.uint32), wire_ref, True)
+    gp.compare("x after apply_delta", x.cpu().numpy(), x_ref, True)
+    gp.compare("x after aggregate_apply", x_one.cpu().numpy(), x_ref1, True)
+    gp.compare("delta bits", dbits.cpu().numpy().view(np.uint32), dbits_ref, True)
+    ctx.destroy()
+
+
 def test_step_host_with_bf16_momentum_and_worker_betas(dl):
     """The host-gradient step slices the momentum arena by its storage type and passes each
     worker's own betas."""
