@@ -294,6 +294,29 @@ int dlion_oracle_aggregate(const dlion_oracle_segment* segs, uint32_t nseg, uint
     return 0;
 }
 
+// The integer the server holds for each coordinate (Section 3.2: the sum of the
+// binary vectors, read as the number of +1 votes, R4) written out as 16-bit
+// values, for worker counts that do not fit the byte output of
+// dlion_oracle_aggregate_apply.  count16[d_pad]; padding is left untouched.
+int dlion_oracle_vote_counts16(const dlion_oracle_segment* segs, uint32_t nseg, uint64_t d_pad,
+                               uint32_t n_workers, const uint32_t* packed, uint16_t* count16) {
+    if (!segs || !packed || !count16 || d_pad % 32 != 0 || n_workers == 0 || n_workers > 65535) return -1;
+    const uint64_t words = d_pad / 32;
+    for (uint32_t s = 0; s < nseg; ++s) {
+        const uint64_t first = segs[s].elem_offset;
+        const uint64_t last = first + segs[s].numel;
+        if (last > d_pad) return -1;
+        for (uint64_t j = first; j < last; ++j) {
+            uint32_t votes = 0;
+            for (uint32_t worker = 0; worker < n_workers; ++worker) {
+                votes += (packed[worker * words + j / 32] >> (j % 32)) & 1u;
+            }
+            count16[j] = static_cast<uint16_t>(votes);
+        }
+    }
+    return 0;
+}
+
 // Worker side, first line of Algorithm 1's loop body: every worker applies the
 // broadcast Delta, x <- x - eps (Delta + lambda x), decoding it from the wire
 // format written by dlion_oracle_aggregate.

@@ -73,6 +73,10 @@ def load(path: Optional[str] = None) -> ctypes.CDLL:
     lib.dlion_oracle_apply_delta.argtypes = [
         ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int,
         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_float]
+    lib.dlion_oracle_vote_counts16.restype = ctypes.c_int
+    lib.dlion_oracle_vote_counts16.argtypes = [
+        ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32,
+        ctypes.c_void_p, ctypes.c_void_p]
     lib.dlion_oracle_global_step.restype = ctypes.c_int
     lib.dlion_oracle_global_step.argtypes = [
         ctypes.POINTER(_Segment), ctypes.c_uint32, ctypes.c_uint64, ctypes.c_uint32, ctypes.c_int,
@@ -204,6 +208,17 @@ def apply_delta(segments, d_pad: int, n_workers: int, mode: int, delta_wire: np.
                                                   _ptr(delta_wire), _ptr(x), lr, weight_decay)
     if rc != 0:
         raise ValueError("dlion_oracle_apply_delta rejected its arguments")
+
+
+def vote_counts16(segments, d_pad: int, n_workers: int, packed: np.ndarray, count16: np.ndarray,
+                  lib: Optional[ctypes.CDLL] = None) -> None:
+    """The number of +1 votes of every parameter as uint16 (any N up to 65535)."""
+    _check(packed, np.uint32, n_workers * d_pad // 32, "packed")
+    _check(count16, np.uint16, d_pad, "count16")
+    rc = (lib or _get()).dlion_oracle_vote_counts16(_segs(segments), len(segments), d_pad, n_workers,
+                                                    _ptr(packed), _ptr(count16))
+    if rc != 0:
+        raise ValueError("dlion_oracle_vote_counts16 rejected its arguments")
 
 
 def global_step(segments, d_pad: int, n_workers: int, g: np.ndarray, m: np.ndarray, x: np.ndarray,

@@ -70,14 +70,20 @@ __device__ __forceinline__ uint32_t lion_coord(float g, float& m, const Betas& k
     return c >= 0.0f ? 1u : 0u;
 }
 
-// The same for two coordinates at once with the packed binary32 instructions of
-// sm_100 (mul/add .rn.f32x2: each element rounded to nearest exactly like the
-// scalar form, so the results are the same bits; half the issue slots).  Returns
-// the two sign bits, coordinate 0 in bit 0.
+// The same for two coordinates at once: the four products come from the packed
+// binary32 multiply of sm_100 (mul.rn.f32x2: each element rounded to nearest exactly
+// like the scalar multiply, half the issue slots), the sums from scalar adds.
+// (The packed ADD must not be used here: fed by a packed multiply, the assembler
+// contracts the pair into a packed fused multiply-add even with contraction
+// switched off -- measured on B200, every mismatch against the scalar form was
+// explained by one fused rounding -- and a fused blend decides other signs.
+// __fadd_rn is never contracted.)  Returns the two sign bits, coordinate 0 in bit 0.
 __device__ __forceinline__ uint32_t lion_pair(float2 g, float2& m, const Betas& k) {
-    const float2 c = __fadd2_rn(__fmul2_rn(make_float2(k.b1, k.b1), m), __fmul2_rn(make_float2(k.om1, k.om1), g));
-    m = __fadd2_rn(__fmul2_rn(make_float2(k.b2, k.b2), m), __fmul2_rn(make_float2(k.om2, k.om2), g));
-    return (c.x >= 0.0f ? 1u : 0u) | (c.y >= 0.0f ? 2u : 0u);
+    const float2 p1 = __fmul2_rn(make_float2(k.b1, k.b1), m), q1 = __fmul2_rn(make_float2(k.om1, k.om1), g);
+    const float2 p2 = __fmul2_rn(make_float2(k.b2, k.b2), m), q2 = __fmul2_rn(make_float2(k.om2, k.om2), g);
+    const float c0 = __fadd_rn(p1.x, q1.x), c1 = __fadd_rn(p1.y, q1.y);
+    m = make_float2(__fadd_rn(p2.x, q2.x), __fadd_rn(p2.y, q2.y));
+    return (c0 >= 0.0f ? 1u : 0u) | (c1 >= 0.0f ? 2u : 0u);
 }
 
 // Four consecutive coordinates held as float4: returns their sign nibble.

@@ -545,9 +545,40 @@ def check_global_lion_definition(lib):
     assert np.array_equal(xa, xb) and np.array_equal(ma, mb)
 
 
+def check_vote_counts16(lib):
+    """16-bit vote counts against a brute-force column sum of the unpacked bits, for worker
+    counts on both sides of one byte; they also agree with the byte counts where those exist
+    and with the count planes of the Averaging message."""
+    rng = np.random.default_rng(16)
+    segs = [(0, 70), (128, 1), (256, 33)]
+    d_pad = 384
+    valid = np.zeros(d_pad, bool)
+    for o, n in segs:
+        valid[o:o + n] = True
+    for N in (1, 3, 255, 256, 257, 1000, 4099):
+        bits = (rng.random((N, d_pad)) < rng.random(d_pad)[None, :]) & valid[None, :]
+        bits[:, 5] = True                      # every worker votes +1: the count is N itself
+        bits[:, 6] = False
+        packed = np.packbits(bits, axis=1, bitorder="little").view(np.uint32).reshape(N, -1).copy()
+        cnt = np.full(d_pad, 0xABCD, np.uint16)
+        orc.vote_counts16(segs, d_pad, N, packed, cnt, lib=lib)
+        P = bits.sum(axis=0)
+        assert np.array_equal(cnt[valid], P[valid].astype(np.uint16)) and cnt[5] == N and cnt[6] == 0
+        assert np.all(cnt[~valid] == 0xABCD)
+        K = orc.delta_planes(N, AVG, lib=lib)
+        wire = np.zeros(K * d_pad // 32, np.uint32)
+        orc.aggregate(segs, d_pad, N, AVG, packed, wire, lib=lib)
+        planes = unpack(wire.reshape(K, -1), d_pad).astype(np.int64)
+        assert np.array_equal((planes << np.arange(K)[:, None]).sum(axis=0)[valid], cnt[valid].astype(np.int64))
+        if N <= 255:
+            c8 = np.zeros(d_pad, np.uint8)
+            orc.aggregate_apply(segs, d_pad, N, MAJ, packed, np.zeros(d_pad, np.float32), 0.1, 0.0, count=c8, lib=lib)
+            assert np.array_equal(c8[valid], cnt[valid].astype(np.uint8))
+
+
 ALL_CHECKS = [check_hand_case, check_sign_of_zero_and_tie, check_delta_is_sign_of_blend,
               check_single_worker_is_lion, check_identical_workers, check_beta_zero_is_signsgd,
               check_equal_betas_is_signum, check_counts_bruteforce, check_x_closed_form,
               check_phase_one_contraction, check_padding_untouched, check_wire_bits,
               check_delta_wire_roundtrip, check_per_worker_betas, check_bf16_momentum_store,
-              check_global_lion_hand_case, check_global_lion_definition]
+              check_global_lion_hand_case, check_global_lion_definition, check_vote_counts16]

@@ -58,6 +58,12 @@ MUTANTS = {
     "global_update_sign": ("x[j] = xo - v3;", "x[j] = xo + v3;"),
     "global_sums_gradients_only": ("const float mt = p1 + q1;                    // the blend each worker would send",
                                    "const float mt = gf;"),
+    "counts16_last_worker_skipped": ("for (uint32_t worker = 0; worker < n_workers; ++worker) {",
+                                     "for (uint32_t worker = 0; worker + 1 < n_workers; ++worker) {"),
+    "counts16_bit_order": ("votes += (packed[worker * words + j / 32] >> (j % 32)) & 1u;",
+                           "votes += (packed[worker * words + j / 32] >> (31 - j % 32)) & 1u;"),
+    "counts16_truncated_to_a_byte": ("count16[j] = static_cast<uint16_t>(votes);",
+                                     "count16[j] = static_cast<uint16_t>(votes & 0xFFu);"),
     "average_down_bits_floor_log": ("while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;",
                                     "while ((2ull << bits) <= static_cast<uint64_t>(n_workers)) ++bits;"),
 }
