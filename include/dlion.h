@@ -134,6 +134,14 @@ dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float
                                    uint32_t* delta_bits_out, uint8_t* count_out,
                                    void* cuda_stream);
 
+/* dlion_aggregate_apply with the vote counts written as 16-bit values, for any N up to
+ * DLION_MAX_WORKERS (the byte output stops at 255): the same vote and the same update.
+ *   count16_out  out, required  [d_pad] uint16: P, the integer in {0..N} the server holds
+ *                (Section 3.2 "Communication Cost"); 8-byte aligned; padding untouched */
+dlion_status dlion_aggregate_apply_counts16(dlion_ctx* ctx, const uint32_t* packed, float* x,
+                                            uint32_t* delta_bits_out, uint16_t* count16_out,
+                                            void* cuda_stream);
+
 /* Server side of Algorithm 1 ALONE (no parameter update): from the N binary
  * vectors, the message the server broadcasts (Section 3.2, "Communication
  * Cost"; Table 1, server->worker column).
@@ -197,6 +205,47 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float*
  *   delta_bits_out  out, nullable  [d_pad/32]: bit = 1 iff the sign is +1 */
 dlion_status dlion_step_global(dlion_ctx* ctx, const void* grads, float* m, float* x,
                                uint32_t* delta_bits_out, void* cuda_stream);
+
+/* ---- Per-tensor mode -------------------------------------------------------------
+ * Algorithm 1 steps a parameter vector x in R^d; in a training framework that vector is
+ * a LIST of separately allocated tensors, with one gradient tensor each.  These calls
+ * step such a list where it lies, without copying it into flat arenas: segment k of the
+ * context's table is tensor k (its elem_offset only numbers its coordinates: the sign
+ * words, Delta bits and the broadcast message stay flat buffers in that numbering).
+ *
+ * dlion_bind_tensors registers the tensors' device addresses:
+ *   grads  host array [N][nseg] of device pointers: worker i's gradient of tensor k at
+ *          grads[i*nseg + k]  (element type as dlion_init's gdtype)
+ *   m      host array [N][nseg]: worker i's momentum of tensor k (float, or bf16 after
+ *          dlion_set_momentum_dtype; set that first)
+ *   x      host array [nseg]: the parameters (float)
+ * A null ARRAY keeps that table as it was bound before (gradients usually move from
+ * step to step, parameters and momenta do not); at least one must be given.  Every
+ * tensor must hold its segment's numel elements and start on a 16-byte boundary
+ * (DLION_EALIGN otherwise; a null tensor pointer is accepted only for numel = 0, else
+ * DLION_EINVAL); nothing is changed when a pointer is rejected.  The tables are copied
+ * into device memory the context owns (allocated on the first call, (2N+1)*nseg
+ * pointers), asynchronously on cuda_stream, in order with the steps issued after it on
+ * the same stream; the host arrays may be reused as soon as the call returns.
+ * Coordinates between one tensor's end and the next segment's start do not exist in
+ * this mode; nothing is read or written outside the tensors. */
+dlion_status dlion_bind_tensors(dlion_ctx* ctx, const void* const* grads, void* const* m,
+                                float* const* x, void* cuda_stream);
+
+/* dlion_worker_step on the bound gradient and momentum tensors (worker = -1: all N;
+ * worker = i: that worker's tensors only, packed then being ITS [d_pad/32] slice).
+ * DLION_ESTATE until gradients and momenta have been bound. */
+dlion_status dlion_worker_step_tensors(dlion_ctx* ctx, int worker, uint32_t* packed, void* cuda_stream);
+
+/* dlion_aggregate_apply on the bound parameter tensors (packed [N][d_pad/32] as there;
+ * delta_bits_out nullable).  DLION_ESTATE until parameters have been bound. */
+dlion_status dlion_aggregate_apply_tensors(dlion_ctx* ctx, const uint32_t* packed,
+                                           uint32_t* delta_bits_out, void* cuda_stream);
+
+/* dlion_apply_delta_sliced (slice_words = 0: dlion_apply_delta) on the bound parameter
+ * tensors.  DLION_ESTATE until parameters have been bound. */
+dlion_status dlion_apply_delta_tensors(dlion_ctx* ctx, const uint32_t* delta_wire, uint64_t slice_words,
+                                       void* cuda_stream);
 
 /* One whole step with the gradients in HOST memory (pinned memory makes the
  * copies asynchronous).  Worker i's gradients are copied to the device while

@@ -50,6 +50,7 @@ __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, ui
     const uint32_t dword = planes_ge<PLANES>(pl, thr) & vmask;
     if (p.delta_bits != nullptr && nbits != 0) p.delta_bits[word_idx] = dword;
     if constexpr (COUNTS) publish_counts<PLANES>(pl, area, lane);
+    float* const xs = p.x_tab != nullptr ? p.x_tab[t.tensor] : p.x;
 #pragma unroll 1
     for (int c = 0; c < 8; ++c) {
         Counts4 k;
@@ -62,9 +63,10 @@ __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, ui
             float delta;
             if constexpr (COUNTS) delta = delta_of_count<PLANES, AVG>(k.c[q], thr, avg_table, p.n_workers);
             else delta = ((dn >> q) & 1u) ? 1.0f : -1.0f;
-            p.x[e + q] = apply_coord(p.x[e + q], delta, p.lr, p.wd);
+            xs[e + q] = apply_coord(xs[e + q], delta, p.lr, p.wd);
             if constexpr (COUNTS) {
                 if (p.count != nullptr) p.count[e + q] = static_cast<uint8_t>(k.c[q]);
+                if (p.count16 != nullptr) p.count16[e + q] = static_cast<uint16_t>(k.c[q]);
             }
         }
     }
@@ -102,9 +104,10 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
         // ---- the votes, all in flight together
         const unsigned long long xe = t.base + warp * kWarpSpan + lane * 4;
         const unsigned long long word_idx = (t.base + warp * kWarpSpan) / 32 + lane;
+        float* const xs = p.x_tab != nullptr ? p.x_tab[t.tensor] : p.x;   // separate tensors, or one arena
         float4 xv[8];
 #pragma unroll
-        for (int c = 0; c < 8; ++c) xv[c] = *(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
+        for (int c = 0; c < 8; ++c) xv[c] = *(reinterpret_cast<const float4*>(xs + xe + c * kChunk));
         if (!have_table) fill_table();
         uint32_t pl[kMaxPlanes];
         count_votes<PLANES>(pl, p.packed + word_idx, p.w_stride, n, true);
@@ -122,6 +125,10 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
                 d2 = delta_of_count<PLANES, AVG>(k.c[2], thr, avg_table, n);
                 d3 = delta_of_count<PLANES, AVG>(k.c[3], thr, avg_table, n);
                 if (p.count != nullptr) *reinterpret_cast<uint32_t*>(p.count + xe + c * kChunk) = pack_counts(k);   // N <= 255 here
+                if (p.count16 != nullptr) {
+                    *reinterpret_cast<uint2*>(p.count16 + xe + c * kChunk) =
+                        make_uint2(k.c[0] | (k.c[1] << 16), k.c[2] | (k.c[3] << 16));
+                }
             } else {
                 const uint32_t dn = my_delta_bits(dword, c, lane);
                 d0 = (dn & 1u) ? 1.0f : -1.0f;
@@ -134,7 +141,7 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
             v.y = apply_coord(v.y, d1, p.lr, p.wd);
             v.z = apply_coord(v.z, d2, p.lr, p.wd);
             v.w = apply_coord(v.w, d3, p.lr, p.wd);
-            *reinterpret_cast<float4*>(p.x + xe + c * kChunk) = v;
+            *reinterpret_cast<float4*>(xs + xe + c * kChunk) = v;
         }
     }
 }
@@ -149,7 +156,7 @@ template <int PLANES>
 cudaError_t launch(const AggParams& p, cudaStream_t s) {
     if (p.ntiles == 0) return cudaSuccess;
     if (p.average) return launch3<PLANES, true, true>(p, s);
-    if (p.count != nullptr) return launch3<PLANES, false, true>(p, s);
+    if (p.count != nullptr || p.count16 != nullptr) return launch3<PLANES, false, true>(p, s);
     return launch3<PLANES, false, false>(p, s);
 }
 

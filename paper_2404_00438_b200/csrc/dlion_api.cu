@@ -15,7 +15,7 @@ using dlion::aligned;
 using dlion::nonneg_finite;
 using dlion::unit_interval;
 
-dlion::Betas betas_of(const dlion_ctx* c) {
+dlion::Betas common_betas(const dlion_ctx* c) {
     dlion::Betas k;
     k.b1 = c->beta1;
     k.om1 = 1.0f - c->beta1;        // formed in binary32, as the contract says
@@ -24,13 +24,63 @@ dlion::Betas betas_of(const dlion_ctx* c) {
     return k;
 }
 
+}  // namespace
+
+namespace dlion {
+
 dlion_status device_ok(const dlion_ctx* c) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
     return dev == c->device ? DLION_OK : DLION_ESTATE;
 }
 
-}  // namespace
+WorkerParams worker_params(const dlion_ctx* ctx, int worker) {
+    WorkerParams p{};
+    p.nseg = ctx->nseg;
+    p.tiles = ctx->tiles_dev;
+    p.flat_d = 0;
+    p.n_workers = worker < 0 ? ctx->n_workers : 1u;
+    p.ntiles = ctx->ntiles;
+    p.d_pad = ctx->d_pad;
+    p.k = common_betas(ctx);
+    p.betas = ctx->betas_dev;
+    p.worker0 = worker < 0 ? 0u : static_cast<uint32_t>(worker);
+    p.m_bf16 = ctx->sdtype == DLION_STATE_BF16 ? 1 : 0;
+    return p;
+}
+
+AggParams agg_params(const dlion_ctx* ctx) {
+    AggParams p{};
+    p.tiles = ctx->tiles_dev;
+    p.flat_d = 0;
+    p.n_workers = ctx->n_workers;
+    p.ntiles = ctx->ntiles;
+    p.w_stride = ctx->d_pad / 32;
+    p.lr = ctx->lr;
+    p.wd = ctx->wd;
+    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    return p;
+}
+
+WireParams wire_params(const dlion_ctx* ctx, uint64_t slice_words) {
+    WireParams p{};
+    p.tiles = ctx->tiles_dev;
+    p.flat_d = 0;
+    p.n_workers = ctx->n_workers;
+    p.ntiles = ctx->ntiles;
+    p.w_stride = ctx->d_pad / 32;
+    p.plane_stride = slice_words != 0 ? slice_words : ctx->d_pad / 32;
+    p.slice_words = slice_words;
+    p.kplanes = dlion_delta_planes(ctx);
+    p.lr = ctx->lr;
+    p.wd = ctx->wd;
+    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    return p;
+}
+
+}  // namespace dlion
+
+using dlion::device_ok;
 
 extern "C" {
 
@@ -139,7 +189,7 @@ dlion_status dlion_set_worker_betas(dlion_ctx* ctx, int worker, float beta1, flo
     if (ds != DLION_OK) return ds;
     if (ctx->betas.empty()) {
         try {
-            ctx->betas.assign(ctx->n_workers, betas_of(ctx));
+            ctx->betas.assign(ctx->n_workers, common_betas(ctx));
         } catch (...) {
             return DLION_ENOMEM;
         }
@@ -171,19 +221,10 @@ dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, vo
     if (!aligned(grads, 16) || !aligned(m, 16) || !aligned(packed, 16)) return DLION_EALIGN;
     const dlion_status ds = device_ok(ctx);
     if (ds != DLION_OK) return ds;
-    dlion::WorkerParams p;
+    dlion::WorkerParams p = dlion::worker_params(ctx, worker);
     p.g = grads;
     p.m = m;
     p.packed = packed;
-    p.tiles = ctx->tiles_dev;
-    p.flat_d = 0;
-    p.n_workers = worker < 0 ? ctx->n_workers : 1u;
-    p.ntiles = ctx->ntiles;
-    p.d_pad = ctx->d_pad;
-    p.k = betas_of(ctx);
-    p.betas = ctx->betas_dev;
-    p.worker0 = worker < 0 ? 0u : static_cast<uint32_t>(worker);
-    p.m_bf16 = ctx->sdtype == DLION_STATE_BF16 ? 1 : 0;
     const cudaError_t e = dlion::launch_worker_step(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
                                                     static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return DLION_ECUDA;
@@ -191,33 +232,50 @@ dlion_status dlion_worker_step(dlion_ctx* ctx, int worker, const void* grads, vo
     return DLION_OK;
 }
 
+namespace {
+dlion_status aggregate_apply_any(dlion_ctx* ctx, const uint32_t* packed, float* x, uint32_t* delta_bits_out,
+                                 uint8_t* count_out, uint16_t* count16_out, void* cuda_stream);
+}
+
 dlion_status dlion_aggregate_apply(dlion_ctx* ctx, const uint32_t* packed, float* x,
                                    uint32_t* delta_bits_out, uint8_t* count_out, void* cuda_stream) {
+    return aggregate_apply_any(ctx, packed, x, delta_bits_out, count_out, nullptr, cuda_stream);
+}
+
+dlion_status dlion_aggregate_apply_counts16(dlion_ctx* ctx, const uint32_t* packed, float* x,
+                                            uint32_t* delta_bits_out, uint16_t* count16_out,
+                                            void* cuda_stream) {
+    if (count16_out == nullptr) return DLION_EINVAL;
+    return aggregate_apply_any(ctx, packed, x, delta_bits_out, nullptr, count16_out, cuda_stream);
+}
+
+}  // extern "C"
+
+namespace {
+dlion_status aggregate_apply_any(dlion_ctx* ctx, const uint32_t* packed, float* x, uint32_t* delta_bits_out,
+                                 uint8_t* count_out, uint16_t* count16_out, void* cuda_stream) {
     if (ctx == nullptr || packed == nullptr || x == nullptr) return DLION_EINVAL;
     if (count_out != nullptr && ctx->n_workers > DLION_MAX_WORKERS_BYTE_COUNTS) return DLION_EINVAL;
-    if (!aligned(packed, 16) || !aligned(x, 16) || !aligned(delta_bits_out, 16) || !aligned(count_out, 4)) {
+    if (!aligned(packed, 16) || !aligned(x, 16) || !aligned(delta_bits_out, 16) || !aligned(count_out, 4) ||
+        !aligned(count16_out, 8)) {
         return DLION_EALIGN;
     }
     const dlion_status ds = device_ok(ctx);
     if (ds != DLION_OK) return ds;
-    dlion::AggParams p;
+    dlion::AggParams p = dlion::agg_params(ctx);
     p.packed = packed;
     p.x = x;
     p.delta_bits = delta_bits_out;
     p.count = count_out;
-    p.tiles = ctx->tiles_dev;
-    p.flat_d = 0;
-    p.n_workers = ctx->n_workers;
-    p.ntiles = ctx->ntiles;
-    p.w_stride = ctx->d_pad / 32;
-    p.lr = ctx->lr;
-    p.wd = ctx->wd;
-    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    p.count16 = count16_out;
     const cudaError_t e = dlion::launch_aggregate_apply(p, ctx->sm_count, static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return DLION_ECUDA;
     if (ctx->ntiles != 0) ctx->launches += 1;
     return DLION_OK;
 }
+}  // namespace
+
+extern "C" {
 
 dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float* x,
                               uint32_t* packed_out, void* cuda_stream) {
@@ -238,7 +296,7 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float*
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
     p.d_pad = ctx->d_pad;
-    p.k = betas_of(ctx);
+    p.k = common_betas(ctx);
     p.betas = ctx->betas_dev;
     p.m_bf16 = ctx->sdtype == DLION_STATE_BF16 ? 1 : 0;
     p.lr = ctx->lr;
@@ -270,7 +328,7 @@ dlion_status dlion_step_global(dlion_ctx* ctx, const void* grads, float* m, floa
     p.n_workers = ctx->n_workers;
     p.ntiles = ctx->ntiles;
     p.d_pad = ctx->d_pad;
-    p.k = betas_of(ctx);
+    p.k = common_betas(ctx);
     p.lr = ctx->lr;
     p.wd = ctx->wd;
     const cudaError_t e = dlion::launch_step_global(p, ctx->gdtype == DLION_GRAD_BF16,

@@ -86,14 +86,6 @@ __device__ __forceinline__ uint32_t lion_pair(float2 g, float2& m, const Betas& 
     return (c0 >= 0.0f ? 1u : 0u) | (c1 >= 0.0f ? 2u : 0u);
 }
 
-// Four consecutive coordinates held as float4: returns their sign nibble.
-__device__ __forceinline__ uint32_t lion_quad(const float4& g, float4& m, const Betas& k) {
-    float2 lo = make_float2(m.x, m.y), hi = make_float2(m.z, m.w);
-    const uint32_t nib = lion_pair(make_float2(g.x, g.y), lo, k) | (lion_pair(make_float2(g.z, g.w), hi, k) << 2);
-    m = make_float4(lo.x, lo.y, hi.x, hi.y);
-    return nib;
-}
-
 // Section 3.2, last equation: x - lr*(Delta + lambda*x).
 __device__ __forceinline__ float apply_coord(float x, float delta, float lr, float wd) {
     return __fsub_rn(x, __fmul_rn(lr, __fadd_rn(delta, __fmul_rn(wd, x))));
@@ -197,9 +189,16 @@ __device__ __forceinline__ uint32_t spread_nibble(uint32_t nibble) {
 }
 
 // ---- launch parameters ----------------------------------------------------
+// Per-tensor pointer tables (dlion_bind_tensors): entry k of a table is tensor k's
+// device address MINUS the byte offset of its first coordinate in the arena numbering,
+// so that table[k] + arena_index * element_size is the element's address and the
+// kernels index exactly as they do into one flat arena.
 struct WorkerParams {
     const void* g;
     void* m;                         // float, or bf16 when m_bf16
+    const void* const* g_tab;        // [n_workers_total][nseg] biased gradient pointers, or null: g is an arena
+    void* const* m_tab;              // likewise for the momentum
+    uint32_t nseg;
     uint32_t* packed;
     const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
     unsigned long long flat_d;
@@ -215,8 +214,10 @@ struct WorkerParams {
 struct AggParams {
     const uint32_t* packed;
     float* x;
+    float* const* x_tab;             // [nseg] biased parameter pointers, or null: x is an arena
     uint32_t* delta_bits;            // nullable
-    uint8_t* count;                  // nullable
+    uint8_t* count;                  // nullable: vote counts, one byte each (N <= 255)
+    uint16_t* count16;               // nullable: vote counts, 16 bits each (any N)
     const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
     unsigned long long flat_d;
     uint32_t n_workers;
@@ -262,6 +263,7 @@ struct WireParams {                  // server-only aggregate / worker-side appl
     uint32_t* wire_out;              // aggregate: the broadcast message
     const uint32_t* wire_in;         // apply: the broadcast message
     float* x;                        // apply: parameters
+    float* const* x_tab;             // apply: [nseg] biased parameter pointers, or null: x is an arena
     const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
     unsigned long long flat_d;
     uint32_t n_workers;
@@ -281,7 +283,7 @@ inline unsigned grid_for(unsigned long long n_items) {
 }
 
 // Host-side launchers (one per .cu file).
-cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s);
+cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s);   // table mode when p.g_tab
 cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s);
 cudaError_t launch_step_fused(const FusedParams& p, bool bf16, int sm_count, cudaStream_t s);
 cudaError_t launch_wire(const WireParams& p, bool apply, cudaStream_t s);

@@ -19,6 +19,11 @@ struct dlion_ctx {
     dlion_sdtype sdtype = DLION_STATE_F32;
     std::vector<dlion::Betas> betas;         // per-worker rows (empty until one is set)
     dlion::Betas* betas_dev = nullptr;
+    // per-tensor pointer tables (dlion_bind_tensors): one device block, g rows first,
+    // then m rows ([n_workers][nseg] each), then the x row ([nseg]); null until bound
+    void** tables_dev = nullptr;
+    std::vector<void*> tables_host;
+    bool bound_g = false, bound_m = false, bound_x = false;
     int device = -1;
     int sm_count = 0;
     uint64_t launches = 0;
@@ -27,3 +32,14 @@ struct dlion_ctx {
     cudaEvent_t consumed[2] = {nullptr, nullptr};
     cudaEvent_t entry = nullptr;
 };
+
+namespace dlion {
+
+// Launch parameters with everything filled in from the context except the caller's
+// pointers (shared by the arena entry points and the per-tensor ones).
+WorkerParams worker_params(const dlion_ctx* c, int worker);
+AggParams agg_params(const dlion_ctx* c);
+WireParams wire_params(const dlion_ctx* c, uint64_t slice_words);
+dlion_status device_ok(const dlion_ctx* c);     // DLION_ESTATE unless the context's device is current
+
+}  // namespace dlion

@@ -115,17 +115,9 @@ dlion_status dlion_aggregate(dlion_ctx* ctx, const uint32_t* packed, uint32_t* d
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
     if (dev != ctx->device) return DLION_ESTATE;
-    dlion::WireParams p{};
+    dlion::WireParams p = dlion::wire_params(ctx, 0);
     p.packed = packed;
     p.wire_out = delta_wire;
-    p.tiles = ctx->tiles_dev;
-    p.flat_d = 0;
-    p.n_workers = ctx->n_workers;
-    p.ntiles = ctx->ntiles;
-    p.w_stride = ctx->d_pad / 32;
-    p.plane_stride = ctx->d_pad / 32;
-    p.kplanes = dlion_delta_planes(ctx);
-    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
     if (dlion::launch_wire(p, false, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
     if (ctx->ntiles != 0) ctx->launches += 1;
     return DLION_OK;
@@ -143,20 +135,9 @@ dlion_status dlion_apply_delta_sliced(dlion_ctx* ctx, const uint32_t* delta_wire
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
     if (dev != ctx->device) return DLION_ESTATE;
-    dlion::WireParams p{};
+    dlion::WireParams p = dlion::wire_params(ctx, slice_words);
     p.wire_in = delta_wire;
     p.x = x;
-    p.tiles = ctx->tiles_dev;
-    p.flat_d = 0;
-    p.n_workers = ctx->n_workers;
-    p.ntiles = ctx->ntiles;
-    p.w_stride = ctx->d_pad / 32;
-    p.plane_stride = slice_words != 0 ? slice_words : ctx->d_pad / 32;
-    p.slice_words = slice_words;
-    p.kplanes = dlion_delta_planes(ctx);
-    p.lr = ctx->lr;
-    p.wd = ctx->wd;
-    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
     if (dlion::launch_wire(p, true, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
     if (ctx->ntiles != 0) ctx->launches += 1;
     return DLION_OK;
@@ -201,6 +182,7 @@ void dlion_destroy(dlion_ctx* ctx) {
     if (ctx == nullptr) return;
     if (ctx->tiles_dev != nullptr) cudaFree(ctx->tiles_dev);
     if (ctx->betas_dev != nullptr) cudaFree(ctx->betas_dev);
+    if (ctx->tables_dev != nullptr) cudaFree(ctx->tables_dev);
     drop_pipeline(ctx);
     delete ctx;
 }

@@ -1,0 +1,135 @@
+// Per-tensor mode of the two-stage path (include/dlion.h): parameters, gradients and
+// momenta that live in separately allocated tensors -- a framework's parameter list --
+// are stepped where they are, through pointer tables, instead of being copied into flat
+// arenas.  The kernels are the arena kernels; only the base address of each stream is
+// looked up per tensor.
+#include <cstring>
+
+#include "dlion_ctx.cuh"
+#include "host_checks.h"
+
+namespace {
+
+using dlion::aligned16;
+
+// Tensor k's address minus the byte offset of its first coordinate in the arena
+// numbering (see WorkerParams).  Plain integer arithmetic: the biased value is only
+// ever used with an index that brings it back inside the tensor.
+void* biased(const void* p, uint64_t elem_offset, size_t elem_size) {
+    return reinterpret_cast<void*>(reinterpret_cast<uintptr_t>(p) - static_cast<uintptr_t>(elem_offset) * elem_size);
+}
+
+}  // namespace
+
+extern "C" {
+
+dlion_status dlion_bind_tensors(dlion_ctx* ctx, const void* const* grads, void* const* m, float* const* x,
+                                void* cuda_stream) {
+    if (ctx == nullptr || (grads == nullptr && m == nullptr && x == nullptr)) return DLION_EINVAL;
+    const dlion_status ds = dlion::device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    const size_t nseg = ctx->nseg, N = ctx->n_workers;
+    const size_t gsz = ctx->gdtype == DLION_GRAD_BF16 ? 2 : 4;
+    const size_t msz = ctx->sdtype == DLION_STATE_BF16 ? 2 : 4;
+    // every pointer is checked before anything changes
+    for (size_t k = 0; k < nseg; ++k) {
+        const bool holds = ctx->segs[k].numel != 0;
+        for (size_t i = 0; i < N; ++i) {
+            if (grads != nullptr && ((holds && grads[i * nseg + k] == nullptr))) return DLION_EINVAL;
+            if (m != nullptr && ((holds && m[i * nseg + k] == nullptr))) return DLION_EINVAL;
+            if (grads != nullptr && !aligned16(grads[i * nseg + k])) return DLION_EALIGN;
+            if (m != nullptr && !aligned16(m[i * nseg + k])) return DLION_EALIGN;
+        }
+        if (x != nullptr && holds && x[k] == nullptr) return DLION_EINVAL;
+        if (x != nullptr && !aligned16(x[k])) return DLION_EALIGN;
+    }
+    const size_t total = (2 * N + 1) * nseg;
+    if (ctx->tables_dev == nullptr) {
+        try {
+            ctx->tables_host.assign(total, nullptr);
+        } catch (...) {
+            return DLION_ENOMEM;
+        }
+        const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->tables_dev), total * sizeof(void*));
+        if (e != cudaSuccess) {
+            ctx->tables_dev = nullptr;
+            ctx->tables_host.clear();
+            return e == cudaErrorMemoryAllocation ? DLION_ENOMEM : DLION_ECUDA;
+        }
+    }
+    void** h = ctx->tables_host.data();
+    for (size_t k = 0; k < nseg; ++k) {
+        const uint64_t off = ctx->segs[k].elem_offset;
+        for (size_t i = 0; i < N; ++i) {
+            if (grads != nullptr) h[i * nseg + k] = biased(grads[i * nseg + k], off, gsz);
+            if (m != nullptr) h[(N + i) * nseg + k] = biased(m[i * nseg + k], off, msz);
+        }
+        if (x != nullptr) h[2 * N * nseg + k] = biased(x[k], off, sizeof(float));
+    }
+    // pageable source: the runtime has taken its copy of the table when this returns,
+    // and the copy itself is ordered on the stream before the steps that follow
+    if (cudaMemcpyAsync(ctx->tables_dev, h, total * sizeof(void*), cudaMemcpyHostToDevice,
+                        static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        return DLION_ECUDA;
+    }
+    ctx->bound_g = ctx->bound_g || grads != nullptr;
+    ctx->bound_m = ctx->bound_m || m != nullptr;
+    ctx->bound_x = ctx->bound_x || x != nullptr;
+    return DLION_OK;
+}
+
+dlion_status dlion_worker_step_tensors(dlion_ctx* ctx, int worker, uint32_t* packed, void* cuda_stream) {
+    if (ctx == nullptr || packed == nullptr) return DLION_EINVAL;
+    if (worker < -1 || worker >= static_cast<int>(ctx->n_workers)) return DLION_EINVAL;
+    if (!ctx->bound_g || !ctx->bound_m) return DLION_ESTATE;
+    if (!aligned16(packed)) return DLION_EALIGN;
+    const dlion_status ds = dlion::device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    dlion::WorkerParams p = dlion::worker_params(ctx, worker);
+    const size_t rows = static_cast<size_t>(ctx->n_workers) * ctx->nseg;
+    p.g_tab = ctx->tables_dev;
+    p.m_tab = ctx->tables_dev + rows;
+    p.packed = packed;
+    if (dlion::launch_worker_step(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
+                                  static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        return DLION_ECUDA;
+    }
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+dlion_status dlion_aggregate_apply_tensors(dlion_ctx* ctx, const uint32_t* packed, uint32_t* delta_bits_out,
+                                           void* cuda_stream) {
+    if (ctx == nullptr || packed == nullptr) return DLION_EINVAL;
+    if (!ctx->bound_x) return DLION_ESTATE;
+    if (!aligned16(packed) || !aligned16(delta_bits_out)) return DLION_EALIGN;
+    const dlion_status ds = dlion::device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    dlion::AggParams p = dlion::agg_params(ctx);
+    p.packed = packed;
+    p.delta_bits = delta_bits_out;
+    p.x_tab = reinterpret_cast<float* const*>(ctx->tables_dev + 2 * static_cast<size_t>(ctx->n_workers) * ctx->nseg);
+    if (dlion::launch_aggregate_apply(p, ctx->sm_count, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        return DLION_ECUDA;
+    }
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+dlion_status dlion_apply_delta_tensors(dlion_ctx* ctx, const uint32_t* delta_wire, uint64_t slice_words,
+                                       void* cuda_stream) {
+    if (ctx == nullptr || delta_wire == nullptr) return DLION_EINVAL;
+    if (slice_words != 0 && (ctx->d_pad / 32) % slice_words != 0) return DLION_EINVAL;
+    if (!ctx->bound_x) return DLION_ESTATE;
+    if (!aligned16(delta_wire)) return DLION_EALIGN;
+    const dlion_status ds = dlion::device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    dlion::WireParams p = dlion::wire_params(ctx, slice_words);
+    p.wire_in = delta_wire;
+    p.x_tab = reinterpret_cast<float* const*>(ctx->tables_dev + 2 * static_cast<size_t>(ctx->n_workers) * ctx->nseg);
+    if (dlion::launch_wire(p, true, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+}  // extern "C"

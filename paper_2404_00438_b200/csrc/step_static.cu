@@ -92,7 +92,7 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
     // The wire buffer keeps the previous call's bits: the worker-side kernel
     // overwrites every word that holds a parameter and the server-side kernel reads
     // no other word, so nothing has to be cleared.
-    dlion::WorkerParams wp;
+    dlion::WorkerParams wp{};
     wp.g = grads;
     wp.m = m;
     wp.packed = wire;
@@ -112,11 +112,12 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
         return DLION_ECUDA;
     }
 
-    dlion::AggParams ap;
+    dlion::AggParams ap{};
     ap.packed = wire;
     ap.x = x;
     ap.delta_bits = nullptr;
     ap.count = nullptr;
+    ap.count16 = nullptr;
     ap.tiles = nullptr;
     ap.flat_d = d;
     ap.n_workers = n_workers;

@@ -70,10 +70,11 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
         const unsigned long long word_idx = (t.base + w0) / 32 + lane;
         const bool live = w0 + lane * 32 < t.valid;                 // my word holds a parameter
 
+        float* const xs = p.x_tab != nullptr ? p.x_tab[t.tensor] : p.x;   // separate tensors, or one arena
         float4 xv[8];
         if (full) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) xv[c] = *(reinterpret_cast<const float4*>(p.x + xe + c * kChunk));
+            for (int c = 0; c < 8; ++c) xv[c] = *(reinterpret_cast<const float4*>(xs + xe + c * kChunk));
         }
         // where my word of plane 0 sits: planes contiguous over all coordinates, or the
         // all-gather order [slice][plane][slice_words] (plane_stride = slice_words then)
@@ -119,10 +120,10 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
                 v.y = apply_coord(v.y, d[1], p.lr, p.wd);
                 v.z = apply_coord(v.z, d[2], p.lr, p.wd);
                 v.w = apply_coord(v.w, d[3], p.lr, p.wd);
-                *reinterpret_cast<float4*>(p.x + e) = v;
+                *reinterpret_cast<float4*>(xs + e) = v;
             } else {
                 for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
-                    p.x[e + q] = apply_coord(p.x[e + q], d[q], p.lr, p.wd);
+                    xs[e + q] = apply_coord(xs[e + q], d[q], p.lr, p.wd);
                 }
             }
         }

@@ -26,10 +26,15 @@ namespace {
 constexpr int kThreads = 256;            // 8 warps x 512 coordinates = one tile
 constexpr int kChunksPerWarp = 4;
 
-// (Parameters are taken by value on purpose: marking them __grid_constant__ measured 6 % slower here.)
-template <bool BF16, bool MB16>
-__global__ void __launch_bounds__(kThreads)
-worker_step_kernel(const WorkerParams p) {
+// TABLE: gradients and momenta are separate tensors reached through per-tensor pointer
+// tables (one extra 8-byte load per stream and block) instead of two flat arenas.
+// Occupancy, measured on the 1.3 B-parameter workload: with fp32 momentum the kernel is
+// bound by DRAM and fastest at the 5 blocks per SM its 48 registers allow (forced to 6
+// or 8 blocks it spills and loses 20-50 %); with bf16 gradients AND bf16 momentum it
+// moves 40 % fewer bytes per coordinate, is bound by instruction issue, and gains from
+// all 8 blocks (32 registers).
+template <bool BF16, bool MB16, bool TABLE>
+__device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
     const unsigned long long w_stride = p.d_pad / 32;
@@ -37,7 +42,15 @@ worker_step_kernel(const WorkerParams p) {
 
     for (unsigned long long tile = blockIdx.x; tile < p.ntiles; tile += gridDim.x) {
         const TileRef t = find_tile(p.tiles, p.flat_d, tile);
-        const unsigned long long wbase = worker * p.d_pad;         // element offset of this worker
+        unsigned long long wbase = worker * p.d_pad;               // element offset of this worker
+        const void* gsrc = p.g;
+        void* mdst = p.m;
+        if constexpr (TABLE) {
+            const unsigned long long row = (p.worker0 + worker) * p.nseg + t.tensor;
+            gsrc = p.g_tab[row];
+            mdst = p.m_tab[row];
+            wbase = 0;
+        }
         const Betas k = betas_of(p.betas, p.k, p.worker0 + worker);
         const uint32_t in_tile = warp * (kChunksPerWarp * kChunk); // first coordinate of this warp
         uint32_t* words = p.packed + worker * w_stride + (t.base + in_tile) / 32;
@@ -47,10 +60,13 @@ worker_step_kernel(const WorkerParams p) {
             if constexpr (BF16 && MB16) {
                 // both streams are bf16: lane l of a 256-coordinate chunk holds coordinates
                 // 8l..8l+7 (one 16-byte access each for g and m), its eight signs are a byte,
-                // and four lanes' bytes make a word (two xor-shuffles)
+                // and four lanes' bytes make a word (two xor-shuffles); the products come
+                // from the packed multiply (this variant is bound by instruction issue:
+                // 20.7 -> 20.0 ms on the 1.3 B-parameter workload; the DRAM-bound fp32-momentum
+                // variants measured 6 % SLOWER with it and keep the scalar form)
                 const unsigned long long e0 = wbase + t.base + in_tile + lane * 8;
-                const uint16_t* gp = static_cast<const uint16_t*>(p.g) + e0;
-                uint16_t* mp = static_cast<uint16_t*>(p.m) + e0;
+                const uint16_t* gp = static_cast<const uint16_t*>(gsrc) + e0;
+                uint16_t* mp = static_cast<uint16_t*>(mdst) + e0;
                 uint4 gv[2], mv[2];
 #pragma unroll
                 for (int u = 0; u < 2; ++u) {
@@ -82,14 +98,17 @@ worker_step_kernel(const WorkerParams p) {
                 float4 g[kChunksPerWarp], m[kChunksPerWarp];
 #pragma unroll
                 for (int u = 0; u < kChunksPerWarp; ++u) {
-                    g[u] = load_grad4<BF16>(p.g, e0 + u * kChunk);
-                    m[u] = load_state4<MB16>(p.m, e0 + u * kChunk);
+                    g[u] = load_grad4<BF16>(gsrc, e0 + u * kChunk);
+                    m[u] = load_state4<MB16>(mdst, e0 + u * kChunk);
                 }
                 uint32_t mine = 0;
 #pragma unroll
                 for (int u = 0; u < kChunksPerWarp; ++u) {
-                    const uint32_t nib = lion_quad(g[u], m[u], k);
-                    store_state4<MB16>(p.m, e0 + u * kChunk, m[u]);
+                    uint32_t nib = lion_coord(g[u].x, m[u].x, k);
+                    nib |= lion_coord(g[u].y, m[u].y, k) << 1;
+                    nib |= lion_coord(g[u].z, m[u].z, k) << 2;
+                    nib |= lion_coord(g[u].w, m[u].w, k) << 3;
+                    store_state4<MB16>(mdst, e0 + u * kChunk, m[u]);
                     const uint32_t w = gather_word(nib, lane);
                     if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
                 }
@@ -106,19 +125,19 @@ worker_step_kernel(const WorkerParams p) {
                 const unsigned long long e = wbase + t.base + j0;
                 uint32_t nib = 0;
                 if (j0 + 4 <= t.valid) {
-                    float4 g = load_grad4<BF16>(p.g, e);
-                    float4 m = load_state4<MB16>(p.m, e);
+                    float4 g = load_grad4<BF16>(gsrc, e);
+                    float4 m = load_state4<MB16>(mdst, e);
                     nib = lion_coord(g.x, m.x, k);
                     nib |= lion_coord(g.y, m.y, k) << 1;
                     nib |= lion_coord(g.z, m.z, k) << 2;
                     nib |= lion_coord(g.w, m.w, k) << 3;
-                    store_state4<MB16>(p.m, e, m);
+                    store_state4<MB16>(mdst, e, m);
                 } else {
                     for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
-                        const float g = load_grad1<BF16>(p.g, e + q);
-                        float m = load_state1<MB16>(p.m, e + q);
+                        const float g = load_grad1<BF16>(gsrc, e + q);
+                        float m = load_state1<MB16>(mdst, e + q);
                         nib |= lion_coord(g, m, k) << q;
-                        store_state1<MB16>(p.m, e + q, m);
+                        store_state1<MB16>(mdst, e + q, m);
                     }
                 }
                 const uint32_t w = gather_word(nib, lane);
@@ -131,11 +150,31 @@ worker_step_kernel(const WorkerParams p) {
     }
 }
 
+// (Parameters are taken by value on purpose: marking them __grid_constant__ measured 6 % slower here.)
+template <bool BF16, bool MB16, bool TABLE>
+__global__ void __launch_bounds__(kThreads)
+worker_step_kernel(const WorkerParams p) {
+    worker_step_body<BF16, MB16, TABLE>(p);
+}
+
+// bf16 gradients and bf16 momentum: 8 blocks per SM (see above)
+template <bool TABLE>
+__global__ void __launch_bounds__(kThreads, 8)
+worker_step_kernel_bf16(const WorkerParams p) {
+    worker_step_body<true, true, TABLE>(p);
+}
+
 template <bool BF16, bool MB16>
 cudaError_t launch(const WorkerParams& p, cudaStream_t s) {
     if (p.ntiles == 0 || p.n_workers == 0) return cudaSuccess;
     const dim3 grid(grid_for(p.ntiles), p.n_workers);               // blocks are dispatched x first: worker-major item order
-    worker_step_kernel<BF16, MB16><<<grid, kThreads, 0, s>>>(p);
+    if constexpr (BF16 && MB16) {
+        if (p.g_tab != nullptr) worker_step_kernel_bf16<true><<<grid, kThreads, 0, s>>>(p);
+        else worker_step_kernel_bf16<false><<<grid, kThreads, 0, s>>>(p);
+    } else {
+        if (p.g_tab != nullptr) worker_step_kernel<BF16, MB16, true><<<grid, kThreads, 0, s>>>(p);
+        else worker_step_kernel<BF16, MB16, false><<<grid, kThreads, 0, s>>>(p);
+    }
     return cudaGetLastError();
 }
 

@@ -24,9 +24,10 @@ OK, EINVAL, EALIGN, ENOMEM, ECUDA, ESTATE = range(6)
 
 EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_set_momentum_dtype",
            "dlion_set_worker_betas", "dlion_worker_step",
-           "dlion_aggregate_apply", "dlion_aggregate", "dlion_apply_delta", "dlion_apply_delta_sliced",
+           "dlion_aggregate_apply", "dlion_aggregate_apply_counts16", "dlion_aggregate", "dlion_apply_delta", "dlion_apply_delta_sliced",
            "dlion_delta_planes",
-           "dlion_step_fused", "dlion_step_global", "dlion_step_host", "dlion_step_static",
+           "dlion_bind_tensors", "dlion_worker_step_tensors", "dlion_aggregate_apply_tensors",
+           "dlion_apply_delta_tensors", "dlion_step_fused", "dlion_step_global", "dlion_step_host", "dlion_step_static",
            "dlion_wire_bytes",
            "dlion_launch_count", "dlion_status_str", "dlion_destroy")
 
@@ -64,6 +65,8 @@ def _load() -> ctypes.CDLL:
     lib.dlion_worker_step.restype = i32
     lib.dlion_aggregate_apply.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.dlion_aggregate_apply.restype = i32
+    lib.dlion_aggregate_apply_counts16.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.dlion_aggregate_apply_counts16.restype = i32
     lib.dlion_aggregate.argtypes = [vp, vp, vp, vp]
     lib.dlion_aggregate.restype = i32
     lib.dlion_apply_delta.argtypes = [vp, vp, vp, vp]
@@ -72,6 +75,14 @@ def _load() -> ctypes.CDLL:
     lib.dlion_apply_delta_sliced.restype = i32
     lib.dlion_delta_planes.argtypes = [vp]
     lib.dlion_delta_planes.restype = u32
+    lib.dlion_bind_tensors.argtypes = [vp, vp, vp, vp, vp]
+    lib.dlion_bind_tensors.restype = i32
+    lib.dlion_worker_step_tensors.argtypes = [vp, i32, vp, vp]
+    lib.dlion_worker_step_tensors.restype = i32
+    lib.dlion_aggregate_apply_tensors.argtypes = [vp, vp, vp, vp]
+    lib.dlion_aggregate_apply_tensors.restype = i32
+    lib.dlion_apply_delta_tensors.argtypes = [vp, vp, u64, vp]
+    lib.dlion_apply_delta_tensors.restype = i32
     lib.dlion_step_fused.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.dlion_step_fused.restype = i32
     lib.dlion_step_global.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -146,6 +157,7 @@ def _stream() -> int:
 
 
 _WORD_DTYPES = tuple(t for t in (torch.int32, getattr(torch, "uint32", None)) if t is not None)
+_HALFWORD_DTYPES = tuple(t for t in (torch.int16, getattr(torch, "uint16", None)) if t is not None)
 _GRAD_DTYPES = {GRAD_F32: (torch.float32,), GRAD_BF16: (torch.bfloat16,)}
 _STATE_DTYPES = {STATE_F32: (torch.float32,), STATE_BF16: (torch.bfloat16,)}
 
@@ -194,6 +206,7 @@ class Dlion:
         self.d_pad, self.n_workers, self.mode, self.gdtype = int(d_pad), int(n_workers), int(mode), int(gdtype)
         self.sdtype = STATE_F32
         self.words = self.d_pad // 32
+        self.numels = [int(n) for _, n in segments]
         self.device_index = torch.cuda.current_device()
 
     def _check(self, st: int, where: str) -> None:
@@ -233,6 +246,16 @@ class Dlion:
         self._check(_lib.dlion_aggregate_apply(self._ctx, _ptr(packed), _ptr(x), _ptr(delta_bits_out),
                                                _ptr(count_out), _stream()), "dlion_aggregate_apply")
 
+    def aggregate_apply_counts16(self, packed: torch.Tensor, x: torch.Tensor,
+                                 delta_bits_out: Optional[torch.Tensor], count16_out: torch.Tensor) -> None:
+        self._t(packed, "packed", _WORD_DTYPES, self.n_workers * self.words)
+        self._t(x, "x", (torch.float32,), self.d_pad)
+        self._t(delta_bits_out, "delta_bits_out", _WORD_DTYPES, self.words, optional=True)
+        self._t(count16_out, "count16_out", _HALFWORD_DTYPES, self.d_pad)
+        self._check(_lib.dlion_aggregate_apply_counts16(self._ctx, _ptr(packed), _ptr(x), _ptr(delta_bits_out),
+                                                        _ptr(count16_out), _stream()),
+                    "dlion_aggregate_apply_counts16")
+
     def aggregate(self, packed: torch.Tensor, delta_wire: torch.Tensor) -> None:
         self._t(packed, "packed", _WORD_DTYPES, self.n_workers * self.words)
         self._t(delta_wire, "delta_wire", _WORD_DTYPES, self.delta_planes() * self.words)
@@ -253,6 +276,57 @@ class Dlion:
 
     def delta_planes(self) -> int:
         return int(_lib.dlion_delta_planes(self._ctx))
+
+    # ---- per-tensor mode: separately allocated tensors stepped in place
+    def _ptr_table(self, rows, name: str, dtypes):
+        """ctypes array of device pointers from a list (or list of lists) of tensors, each
+        checked against its segment's size; the tensors are kept alive by the caller."""
+        flat = [t for row in rows for t in row] if rows and isinstance(rows[0], (list, tuple)) else list(rows)
+        nseg = len(self.numels)
+        if len(flat) % nseg != 0:
+            raise ValueError(f"{name}: {len(flat)} tensors for {nseg} segments")
+        arr = (ctypes.c_void_p * len(flat))()
+        for j, t in enumerate(flat):
+            need = self.numels[j % nseg]
+            if t is None and need == 0:
+                arr[j] = None
+                continue
+            check_tensor(t, f"{name}[{j}]", dtypes, need, self.device_index)
+            arr[j] = t.data_ptr()
+        return arr, len(flat) // nseg
+
+    def bind_tensors(self, grads=None, m=None, x=None) -> None:
+        """``dlion_bind_tensors``: grads and m are [N][nseg] lists of tensors (or flat lists in
+        that order), x an [nseg] list; None keeps the previous binding of that table."""
+        arrs = []
+        for rows, name, dtypes, want in ((grads, "grads", _GRAD_DTYPES[self.gdtype], self.n_workers),
+                                         (m, "m", _STATE_DTYPES[self.sdtype], self.n_workers),
+                                         (x, "x", (torch.float32,), 1)):
+            if rows is None:
+                arrs.append(None)
+                continue
+            arr, got = self._ptr_table(rows, name, dtypes)
+            if got != want:
+                raise ValueError(f"{name}: tensors for {got} workers, expected {want}")
+            arrs.append(arr)
+        self._check(_lib.dlion_bind_tensors(self._ctx, arrs[0], arrs[1], arrs[2], _stream()), "dlion_bind_tensors")
+
+    def worker_step_tensors(self, worker: int, packed: torch.Tensor) -> None:
+        k = self.n_workers if int(worker) < 0 else 1
+        self._t(packed, "packed", _WORD_DTYPES, k * self.words)
+        self._check(_lib.dlion_worker_step_tensors(self._ctx, int(worker), _ptr(packed), _stream()),
+                    "dlion_worker_step_tensors")
+
+    def aggregate_apply_tensors(self, packed: torch.Tensor, delta_bits_out: Optional[torch.Tensor] = None) -> None:
+        self._t(packed, "packed", _WORD_DTYPES, self.n_workers * self.words)
+        self._t(delta_bits_out, "delta_bits_out", _WORD_DTYPES, self.words, optional=True)
+        self._check(_lib.dlion_aggregate_apply_tensors(self._ctx, _ptr(packed), _ptr(delta_bits_out), _stream()),
+                    "dlion_aggregate_apply_tensors")
+
+    def apply_delta_tensors(self, delta_wire: torch.Tensor, slice_words: int = 0) -> None:
+        self._t(delta_wire, "delta_wire", _WORD_DTYPES, self.delta_planes() * self.words)
+        self._check(_lib.dlion_apply_delta_tensors(self._ctx, _ptr(delta_wire), int(slice_words), _stream()),
+                    "dlion_apply_delta_tensors")
 
     def step_fused(self, grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor,
                    packed_out: Optional[torch.Tensor] = None) -> None:

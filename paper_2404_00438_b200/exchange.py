@@ -73,6 +73,21 @@ class DlionKernels:
     def apply_delta_sliced(self, gathered: torch.Tensor, slice_words: int, x: torch.Tensor) -> None:
         self.model.apply_delta_sliced(gathered, slice_words, x)
 
+    # per-tensor mode: this rank's gradient / momentum / parameter tensors, stepped in place
+    def bind_tensors(self, grads=None, m=None, x=None) -> None:
+        """Each a list of this worker's tensors, one per segment (None: keep the binding)."""
+        world = self.model.n_workers
+
+        def rows(own):                                  # only worker `rank`'s row of the table is ever read
+            return None if own is None else [list(own)] * world
+        self.model.bind_tensors(grads=rows(grads), m=rows(m), x=x)
+
+    def worker_step_tensors(self, packed: torch.Tensor) -> None:
+        self.model.worker_step_tensors(self.rank, packed)
+
+    def apply_delta_tensors(self, gathered: torch.Tensor, slice_words: int) -> None:
+        self.model.apply_delta_tensors(gathered, slice_words)
+
 
 class DistributedLion:
     """One rank of Distributed Lion.  ``g``, ``m``, ``x`` have ``d_pad_x`` elements
@@ -138,21 +153,37 @@ class DistributedLion:
         self._all_gather()
         self.kernels.apply_delta_sliced(self.gathered, self.slice_words, x)   # read where the all-gather put them
 
+    def step_tensors(self) -> None:
+        """The same step on the tensors bound with ``kernels.bind_tensors`` (per-tensor mode)."""
+        self.kernels.worker_step_tensors(self.packed)
+        self._all_to_all()
+        self.kernels.aggregate(self.recv, self.wire_slice)
+        self._all_gather()
+        self.kernels.apply_delta_tensors(self.gathered, self.slice_words)
+
 
 class LionOptimizer:
     """Distributed Lion for a list of fp32 parameters on this rank's device.
 
-    The parameters are moved into one flat fp32 arena (each tensor starts on a
-    128-element boundary) and re-pointed at views of it; their ``.grad`` become views
-    of a second flat arena, so backward() accumulates straight into the buffer the
-    worker-side kernel reads.  ``step()`` is one iteration of Algorithm 1 over all
-    of them: one worker-side launch, the exchange, one apply launch.  With a
-    one-rank group this is plain Lion (Eq. 1 of the paper).
+    ``step()`` is one iteration of Algorithm 1 over all of them: one worker-side launch, the
+    exchange, one apply launch.  With a one-rank group this is plain Lion (Eq. 1 of the paper).
+
+    Two ways of reaching the parameters:
+
+    * ``in_place=True``: the parameters and their ``.grad`` tensors stay where the framework
+      allocated them and are stepped there through the library's per-tensor pointer tables
+      (``dlion_bind_tensors``); only the momentum is this object's own.  Gradient addresses
+      are re-read every step, so ``zero_grad(set_to_none=True)`` is fine.  Every parameter
+      and gradient must be contiguous and start on a 16-byte boundary.
+    * ``in_place=False`` (default): the parameters are moved into one flat fp32 arena (each
+      tensor starts on a 128-element boundary) and re-pointed at views of it; their ``.grad``
+      become views of a second flat arena, so backward() accumulates straight into the
+      buffer the worker-side kernel reads.
     """
 
     def __init__(self, params, lr: float = 1e-4, betas: Tuple[float, float] = (0.9, 0.99),
                  weight_decay: float = 0.0, mode: int = 0, group: Optional[dist.ProcessGroup] = None,
-                 kernels=None):
+                 kernels=None, in_place: bool = False, host_staged: bool = False):
         self.params: List[torch.nn.Parameter] = [p for p in params]
         if not self.params:
             raise ValueError("no parameters")
@@ -165,12 +196,22 @@ class LionOptimizer:
             self.segments.append((off, p.numel()))
             off += (p.numel() + ALIGN - 1) // ALIGN * ALIGN
         d_pad = max(off, ALIGN)
+        self.in_place = bool(in_place)
         self.core = DistributedLion(self.segments, d_pad, mode, kernels=kernels, beta1=betas[0], beta2=betas[1],
-                                    lr=lr, weight_decay=weight_decay, gdtype=0, group=group, device=dev)
+                                    lr=lr, weight_decay=weight_decay, gdtype=0, group=group, device=dev,
+                                    host_staged=host_staged)
         n = self.core.d_pad_x
+        self.m = torch.zeros(n, dtype=torch.float32, device=dev)
+        if self.in_place:
+            for p in self.params:
+                if not p.is_contiguous() or p.data_ptr() % 16 != 0:
+                    raise ValueError("in_place needs contiguous parameters that start on a 16-byte boundary")
+            self.x = self.g = None
+            self.core.kernels.bind_tensors(m=[self.m[o:o + k] for o, k in self.segments],
+                                           x=[p.data.view(-1) for p in self.params])
+            return
         self.x = torch.zeros(n, dtype=torch.float32, device=dev)
         self.g = torch.zeros(n, dtype=torch.float32, device=dev)
-        self.m = torch.zeros(n, dtype=torch.float32, device=dev)
         with torch.no_grad():
             for p, (o, k) in zip(self.params, self.segments):
                 self.x[o:o + k].copy_(p.detach().reshape(-1))
@@ -180,11 +221,28 @@ class LionOptimizer:
     def set_lr(self, lr: float) -> None:
         self.core.kernels.set_lr(lr)
 
-    def zero_grad(self) -> None:
+    def zero_grad(self, set_to_none: bool = False) -> None:
+        if self.in_place:
+            for p in self.params:
+                if set_to_none:
+                    p.grad = None
+                elif p.grad is not None:
+                    p.grad.zero_()
+            return
         self.g.zero_()                      # the views stay bound to the arena
 
     @torch.no_grad()
     def step(self) -> None:
+        if self.in_place:
+            grads = []
+            for p in self.params:
+                g = p.grad
+                if g is None or g.dtype != torch.float32 or not g.is_contiguous() or g.data_ptr() % 16 != 0:
+                    raise RuntimeError("in_place needs a contiguous fp32 .grad on a 16-byte boundary for every parameter")
+                grads.append(g.view(-1))
+            self.core.kernels.bind_tensors(grads=grads)
+            self.core.step_tensors()
+            return
         for p, (o, k) in zip(self.params, self.segments):
             if p.grad is None or p.grad.data_ptr() != self.g[o:o + k].data_ptr():
                 raise RuntimeError("a parameter's .grad no longer points into the gradient arena "

@@ -22,7 +22,7 @@ def dl():
 
 def test_exports_match_header(dl):
     header = open(os.path.join(ROOT, "include", "dlion.h")).read()
-    declared = set(re.findall(r"\b(dlion_[a-z_]+)\s*\(", header))
+    declared = set(re.findall(r"\b(dlion_[a-z0-9_]+)\s*\(", header))
     assert declared == set(dl.EXPORTS)
     raw = ctypes.CDLL(dl_build.LIB)
     for name in declared:

@@ -88,3 +88,49 @@ def test_optimizer_wrapper_trains_a_small_model_like_the_oracle():
             assert np.array_equal(flat, want)                   # the model really sees the arena
     finally:
         dist.destroy_process_group()
+
+
+def test_in_place_optimizer_steps_the_models_own_tensors():
+    """in_place=True: parameters and gradients stay where torch allocated them (gradients are
+    even re-allocated every step) and are stepped through the per-tensor pointer tables; the
+    parameters must equal the oracle's x on the same gradients, tensor by tensor."""
+    from paper_2404_00438_b200 import build
+    build.build()
+    from oracle import dlion_oracle as orc
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
+    try:
+        torch.manual_seed(1)
+        model = torch.nn.Sequential(torch.nn.Linear(37, 64), torch.nn.Tanh(), torch.nn.Linear(64, 5000),
+                                    torch.nn.Tanh(), torch.nn.Linear(5000, 3)).to(dev)
+        params = list(model.parameters())
+        ptrs = [p.data_ptr() for p in params]
+        opt = exchange.LionOptimizer(params, lr=1e-2, betas=(0.9, 0.99), weight_decay=0.1, mode=1, in_place=True)
+        D = opt.core.d_pad_x
+        x_ref = np.zeros(D, np.float32)
+        for p, (o, k) in zip(params, opt.segments):
+            x_ref[o:o + k] = p.detach().reshape(-1).cpu().numpy()
+        m_ref = np.zeros((1, D), np.float32)
+        data = torch.randn(16, 37, device=dev)
+        target = torch.randn(16, 3, device=dev)
+        for t in range(3):
+            opt.zero_grad(set_to_none=True)
+            torch.nn.functional.mse_loss(model(data), target).backward()
+            g = np.zeros((1, D), np.float32)
+            for p, (o, k) in zip(params, opt.segments):
+                g[0, o:o + k] = p.grad.reshape(-1).cpu().numpy()
+            opt.step()
+            torch.cuda.synchronize()
+            packed = np.zeros((1, D // 32), np.uint32)
+            orc.worker_step(opt.segments, D, 1, g, m_ref, packed, 0.9, 0.99)
+            orc.aggregate_apply(opt.segments, D, 1, 1, packed, x_ref, 1e-2, 0.1)
+            for p, (o, k) in zip(params, opt.segments):
+                assert np.array_equal(p.detach().reshape(-1).cpu().numpy(), x_ref[o:o + k])
+            assert gp.compare("m", opt.m.cpu().numpy(), m_ref[0], False) == 0
+        assert [p.data_ptr() for p in params] == ptrs            # nothing was moved
+    finally:
+        dist.destroy_process_group()

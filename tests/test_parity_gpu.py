@@ -422,6 +422,36 @@ def test_more_than_255_workers(dl, n, mode):
     ctx.destroy()
 
 
+@pytest.mark.parametrize("n", [3, 200, 255, 256, 300, 1000, 4097])
+@pytest.mark.parametrize("mode", [MAJ, AVG])
+def test_sixteen_bit_counts(dl, n, mode):
+    """dlion_aggregate_apply_counts16 on a ragged table with several tiles: counts equal the
+    oracle's, padding of the count buffer untouched, x as from the plain call."""
+    from oracle import dlion_oracle as orc
+    w = inputs.custom(RAGGED + [2 * 4096 + 5], n, mode, "f32", lr=1e-2, weight_decay=0.5)
+    dev = torch.device("cuda:0")
+    D = w.d_pad
+    rng = np.random.default_rng(n * 2 + mode)
+    valid = np.zeros(D, bool)
+    for off, cnt in w.segments:
+        valid[off:off + cnt] = True
+    bits = (rng.integers(0, 256, (n, D), dtype=np.uint8) < rng.integers(0, 257, D)[None, :]) & valid[None, :]
+    packed_np = np.packbits(bits, axis=1, bitorder="little").view(np.uint32).reshape(n, -1).copy()
+    cnt_ref = np.full(D, 0x5A5A, np.uint16)
+    orc.vote_counts16(w.segments, D, n, packed_np, cnt_ref)
+    x_ref = inputs.fill_x0(w, torch.empty(D)).numpy().copy()
+    orc.aggregate_apply(w.segments, D, n, mode, packed_np, x_ref, w.lr, w.weight_decay)
+    ctx = gp.make_ctx(dl, w)
+    packed = torch.from_numpy(packed_np.view(np.int32)).to(dev)
+    x = inputs.fill_x0(w, torch.empty(D)).to(dev)
+    cnt = torch.full((D,), 0x5A5A, dtype=torch.int16, device=dev)
+    ctx.aggregate_apply_counts16(packed, x, None, cnt)
+    torch.cuda.synchronize()
+    gp.compare("16-bit counts", cnt.cpu().numpy().view(np.uint16), cnt_ref, True)
+    gp.compare("x", x.cpu().numpy(), x_ref, True)
+    ctx.destroy()
+
+
 @pytest.mark.parametrize("n", [8191, 8192, 16383, 16384, 32768, 65535])
 @pytest.mark.parametrize("mode", [MAJ, AVG])
 def test_thirteen_to_sixteen_bit_planes(dl, n, mode):
@@ -471,6 +501,15 @@ def test_thirteen_to_sixteen_bit_planes(dl, n, mode):
     gp.compare("x after apply_delta", x.cpu().numpy(), x_ref, True)
     gp.compare("x after aggregate_apply", x_one.cpu().numpy(), x_ref1, True)
     gp.compare("delta bits", dbits.cpu().numpy().view(np.uint32), dbits_ref, True)
+    # the same call with the vote counts written out, 16 bits each
+    cnt_ref = np.full(D, 0x5A5A, np.uint16)
+    orc.vote_counts16(w.segments, D, n, packed_np, cnt_ref)
+    cnt = torch.full((D,), 0x5A5A, dtype=torch.int16, device=dev)
+    x_cnt = x0.to(dev)
+    ctx.aggregate_apply_counts16(packed, x_cnt, None, cnt)
+    torch.cuda.synchronize()
+    gp.compare("16-bit counts", cnt.cpu().numpy().view(np.uint16), cnt_ref, True)
+    assert torch.equal(x_cnt, x_one)
     ctx.destroy()
 
 
