@@ -189,15 +189,19 @@ __device__ __forceinline__ uint32_t spread_nibble(uint32_t nibble) {
 }
 
 // ---- launch parameters ----------------------------------------------------
-// Per-tensor pointer tables (dlion_bind_tensors): entry k of a table is tensor k's
-// device address MINUS the byte offset of its first coordinate in the arena numbering,
-// so that table[k] + arena_index * element_size is the element's address and the
-// kernels index exactly as they do into one flat arena.
+// Per-tensor tables (dlion_bind_tensors): entry k of a table is the BYTE OFFSET, from the
+// base pointer passed beside the table, of tensor k's storage minus the byte offset of
+// its first coordinate in the arena numbering -- so that base + table[k] +
+// arena_index * element_size is the element's address and the kernels index exactly as
+// they do into one flat arena.  (Offsets from a kernel-argument pointer rather than raw
+// addresses: the compiler then knows the accesses are to global memory and keeps
+// reordering them freely around the shared-memory traffic of the vote; with addresses
+// loaded from a table the Averaging kernel measured 11 % slower, arena mode included.)
 struct WorkerParams {
     const void* g;
     void* m;                         // float, or bf16 when m_bf16
-    const void* const* g_tab;        // [n_workers_total][nseg] biased gradient pointers, or null: g is an arena
-    void* const* m_tab;              // likewise for the momentum
+    const long long* g_off;          // [n_workers_total][nseg] offsets from g, or null: g is an arena
+    const long long* m_off;          // likewise for the momentum, from m
     uint32_t nseg;
     uint32_t* packed;
     const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
@@ -214,7 +218,7 @@ struct WorkerParams {
 struct AggParams {
     const uint32_t* packed;
     float* x;
-    float* const* x_tab;             // [nseg] biased parameter pointers, or null: x is an arena
+    const long long* x_off;          // [nseg] offsets from x, or null: x is an arena
     uint32_t* delta_bits;            // nullable
     uint8_t* count;                  // nullable: vote counts, one byte each (N <= 255)
     uint16_t* count16;               // nullable: vote counts, 16 bits each (any N)
@@ -263,7 +267,7 @@ struct WireParams {                  // server-only aggregate / worker-side appl
     uint32_t* wire_out;              // aggregate: the broadcast message
     const uint32_t* wire_in;         // apply: the broadcast message
     float* x;                        // apply: parameters
-    float* const* x_tab;             // apply: [nseg] biased parameter pointers, or null: x is an arena
+    const long long* x_off;          // apply: [nseg] offsets from x, or null: x is an arena
     const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
     unsigned long long flat_d;
     uint32_t n_workers;
@@ -283,7 +287,7 @@ inline unsigned grid_for(unsigned long long n_items) {
 }
 
 // Host-side launchers (one per .cu file).
-cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s);   // table mode when p.g_tab
+cudaError_t launch_worker_step(const WorkerParams& p, bool bf16, int sm_count, cudaStream_t s);   // table mode when p.g_off
 cudaError_t launch_aggregate_apply(const AggParams& p, int sm_count, cudaStream_t s);
 cudaError_t launch_step_fused(const FusedParams& p, bool bf16, int sm_count, cudaStream_t s);
 cudaError_t launch_wire(const WireParams& p, bool apply, cudaStream_t s);

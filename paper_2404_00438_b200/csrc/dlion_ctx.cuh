@@ -19,10 +19,10 @@ struct dlion_ctx {
     dlion_sdtype sdtype = DLION_STATE_F32;
     std::vector<dlion::Betas> betas;         // per-worker rows (empty until one is set)
     dlion::Betas* betas_dev = nullptr;
-    // per-tensor pointer tables (dlion_bind_tensors): one device block, g rows first,
+    // per-tensor tables (dlion_bind_tensors): one device block, g rows first,
     // then m rows ([n_workers][nseg] each), then the x row ([nseg]); null until bound
-    void** tables_dev = nullptr;
-    std::vector<void*> tables_host;
+    long long* tables_dev = nullptr;         // byte offsets from tables_dev itself (see WorkerParams)
+    std::vector<long long> tables_host;
     bool bound_g = false, bound_m = false, bound_x = false;
     int device = -1;
     int sm_count = 0;

@@ -12,11 +12,13 @@ namespace {
 
 using dlion::aligned16;
 
-// Tensor k's address minus the byte offset of its first coordinate in the arena
-// numbering (see WorkerParams).  Plain integer arithmetic: the biased value is only
-// ever used with an index that brings it back inside the tensor.
-void* biased(const void* p, uint64_t elem_offset, size_t elem_size) {
-    return reinterpret_cast<void*>(reinterpret_cast<uintptr_t>(p) - static_cast<uintptr_t>(elem_offset) * elem_size);
+// Table entry for a tensor: the distance in bytes from `base` to the tensor's storage,
+// minus the byte offset of its first coordinate in the arena numbering (see WorkerParams).
+// Plain integer arithmetic: the biased value is only ever used with an index that brings
+// it back inside the tensor.
+long long entry(const void* tensor, const void* base, uint64_t elem_offset, size_t elem_size) {
+    return static_cast<long long>(reinterpret_cast<uintptr_t>(tensor) - reinterpret_cast<uintptr_t>(base) -
+                                  static_cast<uintptr_t>(elem_offset) * elem_size);
 }
 
 }  // namespace
@@ -46,29 +48,30 @@ dlion_status dlion_bind_tensors(dlion_ctx* ctx, const void* const* grads, void* 
     const size_t total = (2 * N + 1) * nseg;
     if (ctx->tables_dev == nullptr) {
         try {
-            ctx->tables_host.assign(total, nullptr);
+            ctx->tables_host.assign(total, 0);
         } catch (...) {
             return DLION_ENOMEM;
         }
-        const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->tables_dev), total * sizeof(void*));
+        const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->tables_dev), total * sizeof(long long));
         if (e != cudaSuccess) {
             ctx->tables_dev = nullptr;
             ctx->tables_host.clear();
             return e == cudaErrorMemoryAllocation ? DLION_ENOMEM : DLION_ECUDA;
         }
     }
-    void** h = ctx->tables_host.data();
+    long long* h = ctx->tables_host.data();
+    const void* base = ctx->tables_dev;             // the pointer the kernels are given beside each table
     for (size_t k = 0; k < nseg; ++k) {
         const uint64_t off = ctx->segs[k].elem_offset;
         for (size_t i = 0; i < N; ++i) {
-            if (grads != nullptr) h[i * nseg + k] = biased(grads[i * nseg + k], off, gsz);
-            if (m != nullptr) h[(N + i) * nseg + k] = biased(m[i * nseg + k], off, msz);
+            if (grads != nullptr) h[i * nseg + k] = entry(grads[i * nseg + k], base, off, gsz);
+            if (m != nullptr) h[(N + i) * nseg + k] = entry(m[i * nseg + k], base, off, msz);
         }
-        if (x != nullptr) h[2 * N * nseg + k] = biased(x[k], off, sizeof(float));
+        if (x != nullptr) h[2 * N * nseg + k] = entry(x[k], base, off, sizeof(float));
     }
     // pageable source: the runtime has taken its copy of the table when this returns,
     // and the copy itself is ordered on the stream before the steps that follow
-    if (cudaMemcpyAsync(ctx->tables_dev, h, total * sizeof(void*), cudaMemcpyHostToDevice,
+    if (cudaMemcpyAsync(ctx->tables_dev, h, total * sizeof(long long), cudaMemcpyHostToDevice,
                         static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
         return DLION_ECUDA;
     }
@@ -87,8 +90,10 @@ dlion_status dlion_worker_step_tensors(dlion_ctx* ctx, int worker, uint32_t* pac
     if (ds != DLION_OK) return ds;
     dlion::WorkerParams p = dlion::worker_params(ctx, worker);
     const size_t rows = static_cast<size_t>(ctx->n_workers) * ctx->nseg;
-    p.g_tab = ctx->tables_dev;
-    p.m_tab = ctx->tables_dev + rows;
+    p.g = ctx->tables_dev;
+    p.m = ctx->tables_dev;
+    p.g_off = ctx->tables_dev;
+    p.m_off = ctx->tables_dev + rows;
     p.packed = packed;
     if (dlion::launch_worker_step(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
                                   static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
@@ -108,7 +113,8 @@ dlion_status dlion_aggregate_apply_tensors(dlion_ctx* ctx, const uint32_t* packe
     dlion::AggParams p = dlion::agg_params(ctx);
     p.packed = packed;
     p.delta_bits = delta_bits_out;
-    p.x_tab = reinterpret_cast<float* const*>(ctx->tables_dev + 2 * static_cast<size_t>(ctx->n_workers) * ctx->nseg);
+    p.x = reinterpret_cast<float*>(ctx->tables_dev);
+    p.x_off = ctx->tables_dev + 2 * static_cast<size_t>(ctx->n_workers) * ctx->nseg;
     if (dlion::launch_aggregate_apply(p, ctx->sm_count, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
         return DLION_ECUDA;
     }
@@ -126,7 +132,8 @@ dlion_status dlion_apply_delta_tensors(dlion_ctx* ctx, const uint32_t* delta_wir
     if (ds != DLION_OK) return ds;
     dlion::WireParams p = dlion::wire_params(ctx, slice_words);
     p.wire_in = delta_wire;
-    p.x_tab = reinterpret_cast<float* const*>(ctx->tables_dev + 2 * static_cast<size_t>(ctx->n_workers) * ctx->nseg);
+    p.x = reinterpret_cast<float*>(ctx->tables_dev);
+    p.x_off = ctx->tables_dev + 2 * static_cast<size_t>(ctx->n_workers) * ctx->nseg;
     if (dlion::launch_wire(p, true, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
     if (ctx->ntiles != 0) ctx->launches += 1;
     return DLION_OK;

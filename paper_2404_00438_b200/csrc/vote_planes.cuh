@@ -228,21 +228,36 @@ __device__ __forceinline__ void fill_avg_table(float* avg_table, uint32_t n, uin
 
 // Plane capacities the kernels are compiled for: the exact plane count up to 8
 // (N <= 255, where the count matters for speed), then 12 and 16.  A capacity
-// above the needed count only adds zero planes.
+// above the needed count only adds zero planes.  coarse = true (the per-tensor
+// variants, to keep their number down): capacities 4, 8 and 16 only.
 template <typename F>
-inline cudaError_t dispatch_planes(uint32_t n_workers, F&& f) {
-    switch (planes_for(n_workers)) {
-        case 1: return f(std::integral_constant<int, 1>{});
-        case 2: return f(std::integral_constant<int, 2>{});
-        case 3: return f(std::integral_constant<int, 3>{});
-        case 4: return f(std::integral_constant<int, 4>{});
-        case 5: return f(std::integral_constant<int, 5>{});
-        case 6: return f(std::integral_constant<int, 6>{});
-        case 7: return f(std::integral_constant<int, 7>{});
-        case 8: return f(std::integral_constant<int, 8>{});
-        case 9: case 10: case 11: case 12: return f(std::integral_constant<int, 12>{});
-        default: return f(std::integral_constant<int, 16>{});
+inline cudaError_t dispatch_planes(uint32_t n_workers, bool coarse, F&& f) {
+    const uint32_t need = planes_for(n_workers);
+    if (coarse) {
+        if (need <= 4) return f(std::integral_constant<int, 4>{}, std::true_type{});
+        if (need <= 8) return f(std::integral_constant<int, 8>{}, std::true_type{});
+        return f(std::integral_constant<int, 16>{}, std::true_type{});
     }
+    switch (need) {
+        case 1: return f(std::integral_constant<int, 1>{}, std::false_type{});
+        case 2: return f(std::integral_constant<int, 2>{}, std::false_type{});
+        case 3: return f(std::integral_constant<int, 3>{}, std::false_type{});
+        case 4: return f(std::integral_constant<int, 4>{}, std::false_type{});
+        case 5: return f(std::integral_constant<int, 5>{}, std::false_type{});
+        case 6: return f(std::integral_constant<int, 6>{}, std::false_type{});
+        case 7: return f(std::integral_constant<int, 7>{}, std::false_type{});
+        case 8: return f(std::integral_constant<int, 8>{}, std::false_type{});
+        case 9: case 10: case 11: case 12: return f(std::integral_constant<int, 12>{}, std::false_type{});
+        default: return f(std::integral_constant<int, 16>{}, std::false_type{});
+    }
+}
+
+// The base of x for a tile: the arena, or (TABLE) tensor t.tensor's storage through the
+// per-tensor offset table.
+template <bool TABLE>
+__device__ __forceinline__ float* x_base(float* x, const long long* x_off, const TileRef& t) {
+    if constexpr (TABLE) return reinterpret_cast<float*>(reinterpret_cast<char*>(x) + x_off[t.tensor]);
+    return x;
 }
 
 }  // namespace dlion

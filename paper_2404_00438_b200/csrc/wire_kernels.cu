@@ -49,7 +49,7 @@ aggregate_kernel(const __grid_constant__ WireParams p) {
     }
 }
 
-template <int PLANES, bool AVG>
+template <int PLANES, bool AVG, bool TABLE>
 __global__ void __launch_bounds__(kThreads, 6)
 apply_delta_kernel(const __grid_constant__ WireParams p) {
     __shared__ float avg_tables[(AVG && PLANES <= 8) ? kWarps : 1][(AVG && PLANES <= 8) ? 256 : 1];
@@ -70,7 +70,7 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
         const unsigned long long word_idx = (t.base + w0) / 32 + lane;
         const bool live = w0 + lane * 32 < t.valid;                 // my word holds a parameter
 
-        float* const xs = p.x_tab != nullptr ? p.x_tab[t.tensor] : p.x;   // separate tensors, or one arena
+        float* const xs = x_base<TABLE>(p.x, p.x_off, t);   // one arena, or tensor t.tensor's storage
         float4 xv[8];
         if (full) {
 #pragma unroll
@@ -130,14 +130,14 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
     }
 }
 
-template <int PLANES>
+template <int PLANES, bool TABLE>
 cudaError_t launch(const WireParams& p, bool apply, cudaStream_t s) {
     if (p.ntiles == 0) return cudaSuccess;
     const unsigned grid = grid_for(p.ntiles);
     if (apply) {
-        if (p.average) apply_delta_kernel<PLANES, true><<<grid, kThreads, 0, s>>>(p);
-        else apply_delta_kernel<1, false><<<grid, kThreads, 0, s>>>(p);
-    } else {
+        if (p.average) apply_delta_kernel<PLANES, true, TABLE><<<grid, kThreads, 0, s>>>(p);
+        else apply_delta_kernel<1, false, TABLE><<<grid, kThreads, 0, s>>>(p);
+    } else if constexpr (!TABLE) {                       // the vote touches no parameter tensor
         if (p.average) aggregate_kernel<PLANES, true><<<grid, kThreads, 0, s>>>(p);
         else aggregate_kernel<PLANES, false><<<grid, kThreads, 0, s>>>(p);
     }
@@ -153,7 +153,9 @@ uint32_t planes_for(uint32_t n_workers) {      // bit length of N = ceil(log2(N+
 }
 
 cudaError_t launch_wire(const WireParams& p, bool apply, cudaStream_t s) {
-    return dispatch_planes(p.n_workers, [&](auto planes) { return launch<decltype(planes)::value>(p, apply, s); });
+    return dispatch_planes(p.n_workers, apply && p.x_off != nullptr, [&](auto planes, auto table) {
+        return launch<decltype(planes)::value, decltype(table)::value>(p, apply, s);
+    });
 }
 
 }  // namespace dlion

@@ -26,7 +26,7 @@ namespace {
 constexpr int kThreads = 256;            // 8 warps x 512 coordinates = one tile
 constexpr int kChunksPerWarp = 4;
 
-// TABLE: gradients and momenta are separate tensors reached through per-tensor pointer
+// TABLE: gradients and momenta are separate tensors reached through per-tensor offset
 // tables (one extra 8-byte load per stream and block) instead of two flat arenas.
 // Occupancy, measured on the 1.3 B-parameter workload: with fp32 momentum the kernel is
 // bound by DRAM and fastest at the 5 blocks per SM its 48 registers allow (forced to 6
@@ -47,8 +47,8 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
         void* mdst = p.m;
         if constexpr (TABLE) {
             const unsigned long long row = (p.worker0 + worker) * p.nseg + t.tensor;
-            gsrc = p.g_tab[row];
-            mdst = p.m_tab[row];
+            gsrc = static_cast<const char*>(p.g) + p.g_off[row];
+            mdst = static_cast<char*>(p.m) + p.m_off[row];
             wbase = 0;
         }
         const Betas k = betas_of(p.betas, p.k, p.worker0 + worker);
@@ -169,10 +169,10 @@ cudaError_t launch(const WorkerParams& p, cudaStream_t s) {
     if (p.ntiles == 0 || p.n_workers == 0) return cudaSuccess;
     const dim3 grid(grid_for(p.ntiles), p.n_workers);               // blocks are dispatched x first: worker-major item order
     if constexpr (BF16 && MB16) {
-        if (p.g_tab != nullptr) worker_step_kernel_bf16<true><<<grid, kThreads, 0, s>>>(p);
+        if (p.g_off != nullptr) worker_step_kernel_bf16<true><<<grid, kThreads, 0, s>>>(p);
         else worker_step_kernel_bf16<false><<<grid, kThreads, 0, s>>>(p);
     } else {
-        if (p.g_tab != nullptr) worker_step_kernel<BF16, MB16, true><<<grid, kThreads, 0, s>>>(p);
+        if (p.g_off != nullptr) worker_step_kernel<BF16, MB16, true><<<grid, kThreads, 0, s>>>(p);
         else worker_step_kernel<BF16, MB16, false><<<grid, kThreads, 0, s>>>(p);
     }
     return cudaGetLastError();
