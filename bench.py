@@ -240,8 +240,32 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+_JSON_FD = None
+
+
+def keep_stdout_for_the_json_line():
+    """Libraries write banners to stdout (NCCL prints its version when a communicator is
+    created): from here on file descriptor 1 is stderr, and emit() alone writes to the
+    real stdout, so that stdout carries exactly one JSON line."""
+    global _JSON_FD
+    if _JSON_FD is None:
+        sys.stdout.flush()
+        _JSON_FD = os.dup(1)
+        os.dup2(2, 1)
+
+
+def emit(line: dict) -> None:
+    data = (json.dumps(line) + "\n").encode()
+    if _JSON_FD is None:
+        sys.stdout.write(data.decode())
+        sys.stdout.flush()
+    else:
+        os.write(_JSON_FD, data)
+
+
 def run_ours(args):
     import torch.distributed as dist
+    keep_stdout_for_the_json_line()
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
@@ -404,6 +428,15 @@ def run_ours(args):
     units = w.d * N * args.steps * world               # param*worker updates, all ranks
     value = units / (total_ms_max * 1e-3) / 1e9
 
+    # ---- worker = GPU exchange (Algorithm 1's send / broadcast as collectives): on by
+    # default whenever there is more than one rank
+    exch = None
+    if args.exchange or world > 1:
+        try:
+            exch = run_exchange(args, w, mode, dev, world, rank, barrier)
+        except Exception as e:                        # reported, never allowed to take the main line down
+            exch = {"error": f"{type(e).__name__}: {e}"}
+
     # ---- end to end: gradients in pinned host memory, Delta read back
     e2e = None
     if not args.no_e2e:
@@ -483,13 +516,13 @@ def run_ours(args):
                        "per_rank": "each rank steps its own full-size coordinate slab; no collective"},
             "ms_per_step_fresh_grads": fresh_ms, "ms_per_step_graph_replay": graph_ms,
             "roofline": roofline, "roofline_stages": stages, "comparison": comparison,
-            "cpu_baseline": cpu, "e2e": e2e,
+            "exchange": exch, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches, "clocks": clocks,
             "wire_bytes_per_step": {"up_all_workers": up, "down_per_worker": down,
                                     "fp32_gradients_each_way_per_worker": ctx.wire_bytes(2),
                                     "fp32_ring_allreduce_per_gpu": int(2 * (N - 1) / N * 4 * w.d)},
         }
-        print(json.dumps(line), flush=True)
+        emit(line)
     ctx.destroy()
     if world > 1:
         dist.destroy_process_group()
@@ -571,6 +604,56 @@ def run_server_stage(args):
     ctx.destroy()
 
 
+def run_exchange(args, w, mode, dev, world, rank, barrier):
+    """The paper's own deployment, one worker per GPU: worker-side kernel on this rank's
+    gradients, all-to-all of the 1-bit shards, vote on this rank's coordinate slice,
+    all-gather of the broadcast message, apply (exchange.DistributedLion; the collectives
+    are NCCL's).  Times K steps with CUDA events, max over ranks, and reports what crossed
+    the links beside an fp32 all-reduce of the same gradients."""
+    import torch.distributed as dist
+    from paper_2404_00438_b200 import exchange
+    own_group = not dist.is_initialized()
+    if own_group:                                     # one rank: a self-exchange through the same collectives
+        import socket
+        with socket.socket() as s:
+            s.bind(("127.0.0.1", 0))
+            port = s.getsockname()[1]
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
+    try:
+        opt = exchange.DistributedLion(w.segments, w.d_pad, mode, beta1=w.beta1, beta2=w.beta2, lr=w.lr,
+                                       weight_decay=w.weight_decay, gdtype=0 if w.grad_dtype == "f32" else 1,
+                                       device=dev)
+        Dx = opt.d_pad_x
+        g = torch.zeros(Dx, dtype=inputs.grad_torch_dtype(w), device=dev)
+        inputs.fill_grads(w, 0, g[:w.d_pad].unsqueeze(0), workers=[rank % max(w.n_workers, 1)])
+        m = torch.zeros(Dx, device=dev)
+        x = torch.zeros(Dx, device=dev)
+        inputs.fill_x0(w, x[:w.d_pad])
+        stream = torch.cuda.current_stream()
+        for _ in range(3):
+            opt.step(g, m, x)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(args.steps):
+            opt.step(g, m, x)
+        e1.record(stream)
+        barrier()
+        t = torch.tensor([e0.elapsed_time(e1)], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item()) / args.steps
+        sent, received = opt.wire_bytes_per_step()
+        return {"ms_per_step": ms, "value": w.d * world / (ms * 1e-3) / 1e9, "unit": UNIT, "workers": world,
+                "steps": args.steps, "gpu_launches_per_step": 3, "collectives": "all_to_all_single + all_gather_into_tensor (NCCL)",
+                "alltoall_bytes_sent_per_rank": sent, "allgather_bytes_received_per_rank": received,
+                "fp32_ring_allreduce_bytes_per_rank": int(2 * (world - 1) / world * 4 * w.d),
+                "note": "one worker per GPU, d = the workload's parameter count on every rank"}
+    finally:
+        if own_group:
+            dist.destroy_process_group()
+
+
 def run_e2e(args, ctx, w, mode, g, m, x, packed, dev, world, barrier):
     """dlion_step_host: per step, N*D gradient elements host->device, Delta device->host."""
     import torch.distributed as dist
@@ -617,6 +700,8 @@ def main():
                     help="server: time the server-side kernel alone on the workload's wire buffer (1 GPU)")
     ap.add_argument("--graph", action="store_true", help="also time the K steps replayed from one CUDA graph")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--exchange", action="store_true",
+                    help="also time the worker = GPU exchange step (always on with more than one rank)")
     ap.add_argument("--no-extra", action="store_true",
                     help="skip the stages timed after the timed region (other aggregation rule, Global Lion)")
     ap.add_argument("--e2e-steps", type=int, default=2)

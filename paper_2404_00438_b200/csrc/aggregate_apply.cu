@@ -29,7 +29,12 @@ namespace {
 
 constexpr int kThreads = 128;             // 4 warps x 1024 coordinates = one tile
 constexpr int kWarps = kThreads / 32;
-constexpr int kMinBlocks = 6;             // register budget: 6 blocks (24 warps) per SM; 4 once N >= 64
+// Blocks per SM (register budget), measured: 7 up to N = 63 (Averaging at N = 16 on the
+// 1.3 B-parameter workload: 1.96 ms at 6 blocks, 1.89 ms at 7, 2.02 ms at 8, which
+// spills); 5 once N >= 64, where 32 vote words are fetched per round trip (flat 100 M
+// vector, Averaging, N = 64 / 128: 5.9 / 6.15 TB/s at 4 blocks, 6.5 / 6.6 at 5, 6.2 at 6).
+constexpr int kMinBlocks = 7;
+constexpr int kMinBlocksManyWorkers = 5;
 
 __device__ __forceinline__ uint32_t pack_counts(const Counts4& k) {          // N <= 255: one byte each
     return k.c[0] | (k.c[1] << 8) | (k.c[2] << 16) | (k.c[3] << 24);
@@ -77,7 +82,7 @@ __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, ui
 // template parameter, not a run-time test: with the test compiled in, the Averaging
 // kernel measured 7 % slower in arena mode too).
 template <int PLANES, bool AVG, bool COUNTS, bool TABLE>
-__global__ void __launch_bounds__(kThreads, PLANES >= 7 ? 4 : kMinBlocks)
+__global__ void __launch_bounds__(kThreads, PLANES >= 7 ? kMinBlocksManyWorkers : kMinBlocks)
 aggregate_apply_kernel(const __grid_constant__ AggParams p) {
     // Delta of Averaging for every count P, one private copy per warp: it is
     // filled after the tile's first loads are in flight and needs no block barrier.
