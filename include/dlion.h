@@ -247,6 +247,30 @@ dlion_status dlion_aggregate_apply_tensors(dlion_ctx* ctx, const uint32_t* packe
 dlion_status dlion_apply_delta_tensors(dlion_ctx* ctx, const uint32_t* delta_wire, uint64_t slice_words,
                                        void* cuda_stream);
 
+/* ---- Scatter mode: the worker -> server send fused into the worker-side kernel -------
+ * In Algorithm 1 every worker "sends delta_{i,t} to the server".  When the server's work
+ * is spread over S ranks (rank r votes on coordinate slice r), worker i's d bits are cut
+ * into S slices and slice r must reach rank r: an all-to-all.  In this mode the
+ * worker-side kernel stores each sign word straight into the receive buffer of the
+ * slice it belongs to, so that exchange needs no pass of its own.  On a multi-GPU job
+ * the buffers are the peers' memory mapped into this process: the kernel only ever
+ * STORES to them (plain stores; no loads from a peer, no multicast); the caller orders
+ * the vote after every worker's kernel (a barrier) as it would after an all-to-all.
+ *
+ * dlion_bind_scatter (once, outside the step loop; copies synchronously):
+ *   dst          host array [n_dst] of device pointers: dst[r] = receive buffer of slice r,
+ *                uint32 [rows][slice_words], 16-byte aligned
+ *   slice_words  words per slice; n_dst * slice_words must equal d_pad/32
+ *   slot, rows   this worker's row in every receive buffer (slot < rows)
+ * dlion_worker_step_scatter(worker = i): dlion_worker_step for ONE worker (grads and m are
+ * its slices), sign word w of the arena numbering going to
+ * dst[w / slice_words][slot * slice_words + w % slice_words].  Words that hold no
+ * parameter are not written, as in the arena form.  DLION_ESTATE until bound. */
+dlion_status dlion_bind_scatter(dlion_ctx* ctx, uint32_t* const* dst, uint32_t n_dst, uint64_t slice_words,
+                                uint32_t slot, uint32_t rows);
+dlion_status dlion_worker_step_scatter(dlion_ctx* ctx, int worker, const void* grads, void* m,
+                                       void* cuda_stream);
+
 /* One whole step with the gradients in HOST memory (pinned memory makes the
  * copies asynchronous).  Worker i's gradients are copied to the device while
  * worker i-1's are being consumed by the worker-side kernel; after the last

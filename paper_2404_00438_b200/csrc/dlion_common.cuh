@@ -203,6 +203,11 @@ struct WorkerParams {
     const long long* g_off;          // [n_workers_total][nseg] offsets from g, or null: g is an arena
     const long long* m_off;          // likewise for the momentum, from m
     uint32_t nseg;
+    // scatter mode (dlion_worker_step_scatter): the sign words of coordinate slice r go to
+    // the buffer at byte offset dst_off[r] from packed, row `slot` of [rows][slice_words]
+    const long long* dst_off;        // [n_dst] offsets from packed, or null: packed is the [N][d_pad/32] arena
+    unsigned long long slice_words;
+    uint32_t slot;
     uint32_t* packed;
     const TileRow* tiles;            // per-tile rows (device), or null: flat vector of flat_d coordinates
     unsigned long long flat_d;

@@ -24,6 +24,10 @@ struct dlion_ctx {
     long long* tables_dev = nullptr;         // byte offsets from tables_dev itself (see WorkerParams)
     std::vector<long long> tables_host;
     bool bound_g = false, bound_m = false, bound_x = false;
+    // scatter mode (dlion_bind_scatter): byte offsets of the per-slice receive buffers from scatter_dev itself
+    long long* scatter_dev = nullptr;
+    uint32_t scatter_n = 0, scatter_slot = 0;
+    uint64_t scatter_slice_words = 0;
     int device = -1;
     int sm_count = 0;
     uint64_t launches = 0;

@@ -183,6 +183,7 @@ void dlion_destroy(dlion_ctx* ctx) {
     if (ctx->tiles_dev != nullptr) cudaFree(ctx->tiles_dev);
     if (ctx->betas_dev != nullptr) cudaFree(ctx->betas_dev);
     if (ctx->tables_dev != nullptr) cudaFree(ctx->tables_dev);
+    if (ctx->scatter_dev != nullptr) cudaFree(ctx->scatter_dev);
     drop_pipeline(ctx);
     delete ctx;
 }

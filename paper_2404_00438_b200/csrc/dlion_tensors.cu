@@ -1,4 +1,6 @@
-// Per-tensor mode of the two-stage path (include/dlion.h): parameters, gradients and
+// The indirect modes of the two-stage path (include/dlion.h).
+//
+// Per-tensor mode: parameters, gradients and
 // momenta that live in separately allocated tensors -- a framework's parameter list --
 // are stepped where they are, through pointer tables, instead of being copied into flat
 // arenas.  The kernels are the arena kernels; only the base address of each stream is
@@ -135,6 +137,72 @@ dlion_status dlion_apply_delta_tensors(dlion_ctx* ctx, const uint32_t* delta_wir
     p.x = reinterpret_cast<float*>(ctx->tables_dev);
     p.x_off = ctx->tables_dev + 2 * static_cast<size_t>(ctx->n_workers) * ctx->nseg;
     if (dlion::launch_wire(p, true, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
+    if (ctx->ntiles != 0) ctx->launches += 1;
+    return DLION_OK;
+}
+
+// ---- scatter mode: the send of the worker = GPU exchange fused into the worker-side kernel.
+// Instead of one contiguous wire buffer, a worker's sign words are stored straight into
+// one receive buffer per coordinate slice -- on a multi-GPU job the buffers of the ranks
+// that vote on those slices, mapped into this process (plain stores to peer memory, no
+// multicast, no loads from a peer) -- so the all-to-all needs no pass of its own.
+
+dlion_status dlion_bind_scatter(dlion_ctx* ctx, uint32_t* const* dst, uint32_t n_dst, uint64_t slice_words,
+                                uint32_t slot, uint32_t rows) {
+    if (ctx == nullptr || dst == nullptr || n_dst == 0 || slice_words == 0 || slot >= rows) return DLION_EINVAL;
+    if (static_cast<uint64_t>(n_dst) * slice_words != ctx->d_pad / 32) return DLION_EINVAL;   // the slices partition the arena
+    for (uint32_t r = 0; r < n_dst; ++r) {
+        if (dst[r] == nullptr) return DLION_EINVAL;
+        if (!aligned16(dst[r])) return DLION_EALIGN;
+    }
+    const dlion_status ds = dlion::device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    if (ctx->scatter_dev != nullptr && ctx->scatter_n != n_dst) {
+        cudaFree(ctx->scatter_dev);
+        ctx->scatter_dev = nullptr;
+    }
+    if (ctx->scatter_dev == nullptr) {
+        const cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->scatter_dev), n_dst * sizeof(long long));
+        if (e != cudaSuccess) {
+            ctx->scatter_dev = nullptr;
+            return e == cudaErrorMemoryAllocation ? DLION_ENOMEM : DLION_ECUDA;
+        }
+    }
+    std::vector<long long> off;
+    try {
+        off.resize(n_dst);
+    } catch (...) {
+        return DLION_ENOMEM;
+    }
+    for (uint32_t r = 0; r < n_dst; ++r) off[r] = entry(dst[r], ctx->scatter_dev, 0, 1);
+    // synchronous: bound once, outside the step loop
+    if (cudaMemcpy(ctx->scatter_dev, off.data(), n_dst * sizeof(long long), cudaMemcpyHostToDevice) != cudaSuccess) {
+        return DLION_ECUDA;
+    }
+    ctx->scatter_n = n_dst;
+    ctx->scatter_slice_words = slice_words;
+    ctx->scatter_slot = slot;
+    return DLION_OK;
+}
+
+dlion_status dlion_worker_step_scatter(dlion_ctx* ctx, int worker, const void* grads, void* m, void* cuda_stream) {
+    if (ctx == nullptr || grads == nullptr || m == nullptr) return DLION_EINVAL;
+    if (worker < 0 || worker >= static_cast<int>(ctx->n_workers)) return DLION_EINVAL;    // one worker per call
+    if (ctx->scatter_dev == nullptr) return DLION_ESTATE;
+    if (!aligned16(grads) || !aligned16(m)) return DLION_EALIGN;
+    const dlion_status ds = dlion::device_ok(ctx);
+    if (ds != DLION_OK) return ds;
+    dlion::WorkerParams p = dlion::worker_params(ctx, worker);
+    p.g = grads;
+    p.m = m;
+    p.packed = reinterpret_cast<uint32_t*>(ctx->scatter_dev);      // the base the offsets count from
+    p.dst_off = ctx->scatter_dev;
+    p.slice_words = ctx->scatter_slice_words;
+    p.slot = ctx->scatter_slot;
+    if (dlion::launch_worker_step(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
+                                  static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) {
+        return DLION_ECUDA;
+    }
     if (ctx->ntiles != 0) ctx->launches += 1;
     return DLION_OK;
 }

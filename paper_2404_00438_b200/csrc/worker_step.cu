@@ -33,8 +33,26 @@ constexpr int kChunksPerWarp = 4;
 // or 8 blocks it spills and loses 20-50 %); with bf16 gradients AND bf16 momentum it
 // moves 40 % fewer bytes per coordinate, is bound by instruction issue, and gains from
 // all 8 blocks (32 registers).
-template <bool BF16, bool MB16, bool TABLE>
+// Where sign word `wi` (arena word index) of worker `worker` is written: the wire arena,
+// or (SCATTER) row slot + worker of the receive buffer of the coordinate slice it falls in.
+template <bool SCATTER>
+__device__ __forceinline__ uint32_t* word_at(const WorkerParams& p, unsigned long long worker,
+                                             unsigned long long w_stride, unsigned long long wi) {
+    if constexpr (SCATTER) {
+        const unsigned long long r = wi / p.slice_words;
+        uint32_t* buf = reinterpret_cast<uint32_t*>(reinterpret_cast<char*>(p.packed) + p.dst_off[r]);
+        return buf + (p.slot + worker) * p.slice_words + (wi - r * p.slice_words);
+    } else {
+        return p.packed + worker * w_stride + wi;
+    }
+}
+
+// MODE 0: flat arenas.  MODE 1: per-tensor tables for g and m.  MODE 2: flat g and m, sign
+// words scattered to per-slice receive buffers (the send of the exchange fused in).
+template <bool BF16, bool MB16, int MODE>
 __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
+    constexpr bool TABLE = MODE == 1;
+    constexpr bool SCATTER = MODE == 2;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
     const unsigned long long w_stride = p.d_pad / 32;
@@ -53,7 +71,7 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
         }
         const Betas k = betas_of(p.betas, p.k, p.worker0 + worker);
         const uint32_t in_tile = warp * (kChunksPerWarp * kChunk); // first coordinate of this warp
-        uint32_t* words = p.packed + worker * w_stride + (t.base + in_tile) / 32;
+        const unsigned long long word0 = (t.base + in_tile) / 32;  // arena index of this warp's first sign word
 
         if (t.valid == kTile) {
             // ---- full tile: vector path, all loads issued before any use ----
@@ -92,7 +110,7 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
                     if ((lane & 3u) == static_cast<uint32_t>(u)) mine = w;
                 }
                 // lane l (l%4 < 2) holds word l/4 of chunk l%4: word index 8*(l%4) + l/4
-                if ((lane & 3u) < 2u) words[8u * (lane & 3u) + (lane >> 2)] = mine;
+                if ((lane & 3u) < 2u) *word_at<SCATTER>(p, worker, w_stride, word0 + 8u * (lane & 3u) + (lane >> 2)) = mine;
             } else {
                 const unsigned long long e0 = wbase + t.base + in_tile + lane * 4;
                 float4 g[kChunksPerWarp], m[kChunksPerWarp];
@@ -113,7 +131,7 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
                     if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
                 }
                 // lane l (l%8 < 4) holds the word of chunk l%8, group l/8: word index 4*(l%8) + l/8
-                if ((lane & 7u) < kChunksPerWarp) words[4u * (lane & 7u) + (lane >> 3)] = mine;
+                if ((lane & 7u) < kChunksPerWarp) *word_at<SCATTER>(p, worker, w_stride, word0 + 4u * (lane & 7u) + (lane >> 3)) = mine;
             }
         } else {
             // ---- last tile of a segment: per-coordinate guards -------------
@@ -143,7 +161,7 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
                 const uint32_t w = gather_word(nib, lane);
                 // only words that hold at least one parameter are written
                 if ((lane & 7u) == 0 && c0 + (lane >> 3) * 32 < t.valid) {
-                    words[4u * u + (lane >> 3)] = w;
+                    *word_at<SCATTER>(p, worker, w_stride, word0 + 4u * u + (lane >> 3)) = w;
                 }
             }
         }
@@ -151,31 +169,33 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
 }
 
 // (Parameters are taken by value on purpose: marking them __grid_constant__ measured 6 % slower here.)
-template <bool BF16, bool MB16, bool TABLE>
+template <bool BF16, bool MB16, int MODE>
 __global__ void __launch_bounds__(kThreads)
 worker_step_kernel(const WorkerParams p) {
-    worker_step_body<BF16, MB16, TABLE>(p);
+    worker_step_body<BF16, MB16, MODE>(p);
 }
 
 // bf16 gradients and bf16 momentum: 8 blocks per SM (see above)
-template <bool TABLE>
+template <int MODE>
 __global__ void __launch_bounds__(kThreads, 8)
 worker_step_kernel_bf16(const WorkerParams p) {
-    worker_step_body<true, true, TABLE>(p);
+    worker_step_body<true, true, MODE>(p);
+}
+
+template <bool BF16, bool MB16, int MODE>
+cudaError_t launch_mode(const WorkerParams& p, const dim3 grid, cudaStream_t s) {
+    if constexpr (BF16 && MB16) worker_step_kernel_bf16<MODE><<<grid, kThreads, 0, s>>>(p);
+    else worker_step_kernel<BF16, MB16, MODE><<<grid, kThreads, 0, s>>>(p);
+    return cudaGetLastError();
 }
 
 template <bool BF16, bool MB16>
 cudaError_t launch(const WorkerParams& p, cudaStream_t s) {
     if (p.ntiles == 0 || p.n_workers == 0) return cudaSuccess;
     const dim3 grid(grid_for(p.ntiles), p.n_workers);               // blocks are dispatched x first: worker-major item order
-    if constexpr (BF16 && MB16) {
-        if (p.g_off != nullptr) worker_step_kernel_bf16<true><<<grid, kThreads, 0, s>>>(p);
-        else worker_step_kernel_bf16<false><<<grid, kThreads, 0, s>>>(p);
-    } else {
-        if (p.g_off != nullptr) worker_step_kernel<BF16, MB16, true><<<grid, kThreads, 0, s>>>(p);
-        else worker_step_kernel<BF16, MB16, false><<<grid, kThreads, 0, s>>>(p);
-    }
-    return cudaGetLastError();
+    if (p.g_off != nullptr) return launch_mode<BF16, MB16, 1>(p, grid, s);
+    if (p.dst_off != nullptr) return launch_mode<BF16, MB16, 2>(p, grid, s);
+    return launch_mode<BF16, MB16, 0>(p, grid, s);
 }
 
 }  // namespace

@@ -27,7 +27,7 @@ EXPORTS = ("dlion_check_layout", "dlion_init", "dlion_set_lr", "dlion_set_moment
            "dlion_aggregate_apply", "dlion_aggregate_apply_counts16", "dlion_aggregate", "dlion_apply_delta", "dlion_apply_delta_sliced",
            "dlion_delta_planes",
            "dlion_bind_tensors", "dlion_worker_step_tensors", "dlion_aggregate_apply_tensors",
-           "dlion_apply_delta_tensors", "dlion_step_fused", "dlion_step_global", "dlion_step_host", "dlion_step_static",
+           "dlion_apply_delta_tensors", "dlion_bind_scatter", "dlion_worker_step_scatter", "dlion_step_fused", "dlion_step_global", "dlion_step_host", "dlion_step_static",
            "dlion_wire_bytes",
            "dlion_launch_count", "dlion_status_str", "dlion_destroy")
 
@@ -83,6 +83,10 @@ def _load() -> ctypes.CDLL:
     lib.dlion_aggregate_apply_tensors.restype = i32
     lib.dlion_apply_delta_tensors.argtypes = [vp, vp, u64, vp]
     lib.dlion_apply_delta_tensors.restype = i32
+    lib.dlion_bind_scatter.argtypes = [vp, vp, u32, u64, u32, u32]
+    lib.dlion_bind_scatter.restype = i32
+    lib.dlion_worker_step_scatter.argtypes = [vp, i32, vp, vp, vp]
+    lib.dlion_worker_step_scatter.restype = i32
     lib.dlion_step_fused.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.dlion_step_fused.restype = i32
     lib.dlion_step_global.argtypes = [vp, vp, vp, vp, vp, vp]
@@ -327,6 +331,28 @@ class Dlion:
         self._t(delta_wire, "delta_wire", _WORD_DTYPES, self.delta_planes() * self.words)
         self._check(_lib.dlion_apply_delta_tensors(self._ctx, _ptr(delta_wire), int(slice_words), _stream()),
                     "dlion_apply_delta_tensors")
+
+    # ---- scatter mode: sign words stored straight into per-slice receive buffers
+    def bind_scatter(self, dst, slice_words: int, slot: int, rows: int) -> None:
+        """``dlion_bind_scatter``: ``dst`` is a list with one entry per coordinate slice, each a
+        tensor [rows, slice_words] of int32 on this device, or an integer device address (a
+        peer's buffer mapped into this process; its extent cannot be checked here)."""
+        arr = (ctypes.c_void_p * len(dst))()
+        for r, t in enumerate(dst):
+            if isinstance(t, int):
+                arr[r] = t
+            else:
+                check_tensor(t, f"dst[{r}]", _WORD_DTYPES, int(rows) * int(slice_words), self.device_index)
+                arr[r] = t.data_ptr()
+        self._scatter_keepalive = [t for t in dst if not isinstance(t, int)]
+        self._check(_lib.dlion_bind_scatter(self._ctx, arr, len(dst), int(slice_words), int(slot), int(rows)),
+                    "dlion_bind_scatter")
+
+    def worker_step_scatter(self, worker: int, grads: torch.Tensor, m: torch.Tensor) -> None:
+        self._t(grads, "grads", _GRAD_DTYPES[self.gdtype], self.d_pad)
+        self._t(m, "m", _STATE_DTYPES[self.sdtype], self.d_pad)
+        self._check(_lib.dlion_worker_step_scatter(self._ctx, int(worker), _ptr(grads), _ptr(m), _stream()),
+                    "dlion_worker_step_scatter")
 
     def step_fused(self, grads: torch.Tensor, m: torch.Tensor, x: torch.Tensor,
                    packed_out: Optional[torch.Tensor] = None) -> None:

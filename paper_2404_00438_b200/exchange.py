@@ -88,6 +88,13 @@ class DlionKernels:
     def apply_delta_tensors(self, gathered: torch.Tensor, slice_words: int) -> None:
         self.model.apply_delta_tensors(gathered, slice_words)
 
+    # scatter mode: the worker-side kernel stores its sign words into the ranks' receive buffers
+    def bind_scatter(self, receive_buffers, slice_words: int, rows: int) -> None:
+        self.model.bind_scatter(receive_buffers, slice_words, slot=self.rank, rows=rows)
+
+    def worker_step_scatter(self, g: torch.Tensor, m: torch.Tensor) -> None:
+        self.model.worker_step_scatter(self.rank, g, m)
+
 
 class DistributedLion:
     """One rank of Distributed Lion.  ``g``, ``m``, ``x`` have ``d_pad_x`` elements
@@ -95,12 +102,23 @@ class DistributedLion:
 
     ``host_staged = True`` routes the two collectives through pinned host buffers (for
     process groups that only move host memory, such as gloo); the default hands the device
-    buffers to the group's backend (NCCL)."""
+    buffers to the group's backend (NCCL).
+
+    ``fused_send = True`` replaces the all-to-all: the receive buffer is allocated as
+    symmetric memory (every rank's buffer mapped into every process), the worker-side
+    kernel stores each sign word straight into the buffer of the rank that votes on it
+    (``dlion_worker_step_scatter``: plain stores to peer memory, no multicast), and a
+    barrier of the group orders the votes after all the stores.  The next step's stores
+    cannot overtake this step's votes: a rank leaves the all-gather only after every rank
+    has produced its part of the message, i.e. has finished reading its receive buffer.
+    Exercised with one rank and, with the ranks emulated as buffers on one GPU, in the
+    tests; it has not run on several GPUs."""
 
     def __init__(self, segments: Sequence[Tuple[int, int]], d_pad: int, mode: int, kernels=None,
                  beta1: float = 0.9, beta2: float = 0.99, lr: float = 1e-4, weight_decay: float = 0.0,
                  gdtype: int = 0, group: Optional[dist.ProcessGroup] = None,
-                 device: Optional[torch.device] = None, host_staged: bool = False):
+                 device: Optional[torch.device] = None, host_staged: bool = False,
+                 fused_send: bool = False):
         self.group = group
         self.world = dist.get_world_size(group)
         self.rank = dist.get_rank(group)
@@ -118,6 +136,16 @@ class DistributedLion:
         self.wire_slice = torch.zeros(self.k, self.slice_words, **z)         # message for my slice
         # every slice's message, in the order the all-gather delivers them: [slice][plane][word]
         self.gathered = torch.zeros(self.world, self.k, self.slice_words, **z)
+        self.fused_send = bool(fused_send)
+        if self.fused_send:
+            if host_staged:
+                raise ValueError("fused_send stores into peer device memory: it cannot be host-staged")
+            import torch.distributed._symmetric_memory as symm_mem
+            self.recv = symm_mem.empty((self.world, self.slice_words), dtype=torch.int32, device=dev)
+            self.recv.zero_()
+            self._symm = symm_mem.rendezvous(self.recv, group if group is not None else dist.group.WORLD)
+            self.kernels.bind_scatter([int(p) for p in self._symm.buffer_ptrs], self.slice_words, rows=self.world)
+            dist.barrier(group=self.group)              # every buffer is zeroed before anyone stores into it
         self.host_staged = bool(host_staged) and dev.type == "cuda"
         if self.host_staged:
             h = dict(dtype=torch.int32, pin_memory=True)
@@ -147,8 +175,12 @@ class DistributedLion:
         self.gathered.view(-1).copy_(self.h_gathered, non_blocking=True)
 
     def step(self, g: torch.Tensor, m: torch.Tensor, x: torch.Tensor) -> None:
-        self.kernels.worker_step(g, m, self.packed)
-        self._all_to_all()
+        if self.fused_send:
+            self.kernels.worker_step_scatter(g, m)      # the send is part of the kernel
+            dist.barrier(group=self.group)              # all stores have landed before anyone votes
+        else:
+            self.kernels.worker_step(g, m, self.packed)
+            self._all_to_all()
         self.kernels.aggregate(self.recv, self.wire_slice)
         self._all_gather()
         self.kernels.apply_delta_sliced(self.gathered, self.slice_words, x)   # read where the all-gather put them

@@ -134,3 +134,42 @@ def test_in_place_optimizer_steps_the_models_own_tensors():
         assert [p.data_ptr() for p in params] == ptrs            # nothing was moved
     finally:
         dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("mode", [inputs.MAJORITY, inputs.AVERAGE])
+def test_fused_send_with_one_rank_matches_oracle(mode):
+    """fused_send=True (receive buffer in symmetric memory, sign words stored by the
+    worker-side kernel, barrier instead of the all-to-all) through a one-rank NCCL group.
+    Skipped where this torch build cannot set up symmetric memory on the box."""
+    from paper_2404_00438_b200 import build
+    build.build()
+    from oracle import dlion_oracle as orc
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda:0")
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
+    try:
+        w = inputs.custom([70000, 333, 4097], 1, mode, "bf16", scale=1e-3, lr=1e-3, weight_decay=1.0)
+        try:
+            opt = exchange.DistributedLion(w.segments, w.d_pad, mode, beta1=w.beta1, beta2=w.beta2, lr=w.lr,
+                                           weight_decay=w.weight_decay, gdtype=1, fused_send=True)
+        except (ImportError, RuntimeError, AttributeError) as e:
+            pytest.skip(f"symmetric memory is not available here: {e}")
+        D = opt.d_pad_x
+        x0 = inputs.fill_x0(w, torch.empty(D))
+        x, m = x0.to(dev), torch.zeros(D, device=dev)
+        x_ref, m_ref = x0.numpy().copy(), np.zeros((1, D), np.float32)
+        for t in range(3):
+            g = inputs.fill_grads(w, t, torch.empty(1, D, dtype=torch.bfloat16))
+            opt.step(g[0].to(dev), m, x)
+            torch.cuda.synchronize()
+            packed = np.zeros((1, D // 32), np.uint32)
+            orc.worker_step(w.segments, D, 1, inputs.as_numpy_grads(g), m_ref, packed, w.beta1, w.beta2)
+            orc.aggregate_apply(w.segments, D, 1, mode, packed, x_ref, w.lr, w.weight_decay)
+            gp.compare("receive buffer", opt.recv.cpu().numpy().view(np.uint32), packed, True)
+            assert gp.compare("m", m.cpu().numpy(), m_ref[0], False) == 0
+            assert gp.compare("x", x.cpu().numpy(), x_ref, False) == 0
+    finally:
+        dist.destroy_process_group()
