@@ -12,27 +12,33 @@
 // a compact window that sweeps the arenas front to back, which measured 12 %
 // faster on B200 than a persistent grid striding over the items (6.9 vs 6.2
 // TB/s), and the same as a persistent grid drawing items from an atomic
-// counter.  Inside a tile each warp owns 512 consecutive
-// coordinates as four 128-coordinate chunks; lane l of a chunk holds coordinates
+// counter.  Inside a tile each of the block's four warps owns 1024 consecutive
+// coordinates as eight 128-coordinate chunks; lane l of a chunk holds coordinates
 // 4l..4l+3, so every load and store instruction of a warp is one contiguous run
 // (16 B per lane for fp32, 8 B per lane for bf16 gradients).  Eight lanes'
-// nibbles are merged into a word by three xor-shuffles, and the warp's 16 words
-// leave as one 64-byte run.
+// nibbles are merged into a word by three xor-shuffles, and the warp's 32 words
+// leave as one 128-byte run, one word per lane.  A thread thus carries 32
+// coordinates: the per-block work that does not scale with coordinates (tile
+// lookup, 64-bit index arithmetic, beta row) is paid once per 32, not per 16 --
+// against 256-thread blocks with 16 coordinates per thread this measured +0.3 to
+// +1.4 % for the DRAM-bound variants and +10 % for the bf16/bf16 variant below.
 #include "dlion_common.cuh"
 
 namespace dlion {
 namespace {
 
-constexpr int kThreads = 256;            // 8 warps x 512 coordinates = one tile
-constexpr int kChunksPerWarp = 4;
+constexpr int kThreads = 128;            // 4 warps x 1024 coordinates = one tile
+constexpr int kChunksPerWarp = 8;        // 128-coordinate chunks per warp
+constexpr int kWideChunks = 4;           // 256-coordinate chunks per warp (bf16/bf16 path)
 
 // TABLE: gradients and momenta are separate tensors reached through per-tensor offset
 // tables (one extra 8-byte load per stream and block) instead of two flat arenas.
 // Occupancy, measured on the 1.3 B-parameter workload: with fp32 momentum the kernel is
-// bound by DRAM and fastest at the 5 blocks per SM its 48 registers allow (forced to 6
-// or 8 blocks it spills and loses 20-50 %); with bf16 gradients AND bf16 momentum it
-// moves 40 % fewer bytes per coordinate, is bound by instruction issue, and gains from
-// all 8 blocks (32 registers).
+// bound by DRAM and fastest with the register allocation the compiler picks unprompted
+// (80-96 registers, 5 blocks per SM; forced to more blocks it spills and loses up to
+// 50 %); with bf16 gradients AND bf16 momentum it moves 40 % fewer bytes per coordinate,
+// leans on instruction issue, and is fastest at 10 blocks per SM (48 registers; 18.5 ms
+// against 19.1 at 9 and 8 blocks and 20.7 at 11 and 12, which spill).
 // Where sign word `wi` (arena word index) of worker `worker` is written: the wire arena,
 // or (SCATTER) row slot + worker of the receive buffer of the coordinate slice it falls in.
 template <bool SCATTER>
@@ -85,15 +91,15 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
                 const unsigned long long e0 = wbase + t.base + in_tile + lane * 8;
                 const uint16_t* gp = static_cast<const uint16_t*>(gsrc) + e0;
                 uint16_t* mp = static_cast<uint16_t*>(mdst) + e0;
-                uint4 gv[2], mv[2];
+                uint4 gv[kWideChunks], mv[kWideChunks];
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
+                for (int u = 0; u < kWideChunks; ++u) {
                     gv[u] = *reinterpret_cast<const uint4*>(gp + u * 2 * kChunk);
                     mv[u] = *reinterpret_cast<const uint4*>(mp + u * 2 * kChunk);
                 }
                 uint32_t mine = 0;
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
+                for (int u = 0; u < kWideChunks; ++u) {
                     const uint32_t gw[4] = {gv[u].x, gv[u].y, gv[u].z, gv[u].w};
                     const uint32_t mw[4] = {mv[u].x, mv[u].y, mv[u].z, mv[u].w};
                     uint32_t out[4], byte = 0;
@@ -109,8 +115,8 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
                     w |= __shfl_xor_sync(kFull, w, 2);
                     if ((lane & 3u) == static_cast<uint32_t>(u)) mine = w;
                 }
-                // lane l (l%4 < 2) holds word l/4 of chunk l%4: word index 8*(l%4) + l/4
-                if ((lane & 3u) < 2u) *word_at<SCATTER>(p, worker, w_stride, word0 + 8u * (lane & 3u) + (lane >> 2)) = mine;
+                // lane l holds word l/4 of chunk l%4: word index 8*(l%4) + l/4
+                *word_at<SCATTER>(p, worker, w_stride, word0 + 8u * (lane & 3u) + (lane >> 2)) = mine;
             } else {
                 const unsigned long long e0 = wbase + t.base + in_tile + lane * 4;
                 float4 g[kChunksPerWarp], m[kChunksPerWarp];
@@ -130,8 +136,8 @@ __device__ __forceinline__ void worker_step_body(const WorkerParams& p) {
                     const uint32_t w = gather_word(nib, lane);
                     if ((lane & 7u) == static_cast<uint32_t>(u)) mine = w;
                 }
-                // lane l (l%8 < 4) holds the word of chunk l%8, group l/8: word index 4*(l%8) + l/8
-                if ((lane & 7u) < kChunksPerWarp) *word_at<SCATTER>(p, worker, w_stride, word0 + 4u * (lane & 7u) + (lane >> 3)) = mine;
+                // lane l holds the word of chunk l%8, group l/8: word index 4*(l%8) + l/8
+                *word_at<SCATTER>(p, worker, w_stride, word0 + 4u * (lane & 7u) + (lane >> 3)) = mine;
             }
         } else {
             // ---- last tile of a segment: per-coordinate guards -------------
@@ -175,9 +181,9 @@ worker_step_kernel(const WorkerParams p) {
     worker_step_body<BF16, MB16, MODE>(p);
 }
 
-// bf16 gradients and bf16 momentum: 8 blocks per SM (see above)
+// bf16 gradients and bf16 momentum: 10 blocks per SM (see above)
 template <int MODE>
-__global__ void __launch_bounds__(kThreads, 8)
+__global__ void __launch_bounds__(kThreads, 10)
 worker_step_kernel_bf16(const WorkerParams p) {
     worker_step_body<true, true, MODE>(p);
 }
