@@ -36,6 +36,11 @@
 //   R5  delta_{i,t} uses the OLD momentum m_{i,t} (both equations carry the
 //       subscript t on their right-hand sides).
 //   R6  Averaging: Delta = (float)(2P-N) / (float)N, IEEE division.
+//   R3' (optional, mode DLION_ORACLE_MAJORITY_TERNARY) the other reading of an
+//       even-N tie: the three-valued sign the appendix's lemma works with,
+//       sign(0) = 0, so S = 0 gives Delta = 0 and the step is pure weight decay
+//       there.  Delta then has three values and takes two bits on the wire,
+//       sent as the integer Delta + 1 in {0, 1, 2} (two planes, like a count).
 //
 // Parity status: every function below is pinned by tests/test_oracle_pins.py
 // (special cases N=1, identical workers, beta=0, beta1=beta2, brute-force vote
@@ -63,7 +68,11 @@ struct dlion_oracle_segment {
     uint64_t numel;
 };
 
-enum { DLION_ORACLE_MAJORITY = 0, DLION_ORACLE_AVERAGE = 1 };
+enum { DLION_ORACLE_MAJORITY = 0, DLION_ORACLE_AVERAGE = 1, DLION_ORACLE_MAJORITY_TERNARY = 2 };
+
+static bool known_mode(int mode) {
+    return mode == DLION_ORACLE_MAJORITY || mode == DLION_ORACLE_AVERAGE || mode == DLION_ORACLE_MAJORITY_TERNARY;
+}
 enum { DLION_ORACLE_GRAD_F32 = 0, DLION_ORACLE_GRAD_BF16 = 1 };
 enum { DLION_ORACLE_STATE_F32 = 0, DLION_ORACLE_STATE_BF16 = 1 };
 
@@ -196,7 +205,7 @@ int dlion_oracle_aggregate_apply(const dlion_oracle_segment* segs, uint32_t nseg
                                  float lr, float weight_decay, int nthreads) {
     if (!segs || !packed || !x || d_pad % 32 != 0 || n_workers == 0) return -1;
     if (count && n_workers > 255) return -1;
-    if (mode != DLION_ORACLE_MAJORITY && mode != DLION_ORACLE_AVERAGE) return -1;
+    if (!known_mode(mode)) return -1;
     const uint64_t W = d_pad / 32;
     const int32_t N = static_cast<int32_t>(n_workers);
     (void)nthreads;
@@ -221,6 +230,8 @@ int dlion_oracle_aggregate_apply(const dlion_oracle_segment* segs, uint32_t nseg
                 float Delta;
                 if (mode == DLION_ORACLE_AVERAGE) {
                     Delta = static_cast<float>(S) / static_cast<float>(N);   // R6
+                } else if (mode == DLION_ORACLE_MAJORITY_TERNARY) {
+                    Delta = (S > 0) ? 1.0f : ((S < 0) ? -1.0f : 0.0f);       // R3': sign(0) = 0
                 } else {
                     Delta = (S >= 0) ? 1.0f : -1.0f;             // R2, R3
                 }
@@ -243,6 +254,7 @@ int dlion_oracle_aggregate_apply(const dlion_oracle_segment* segs, uint32_t nseg
 // (Section 3.2 "Communication Cost"; the paper rounds this to log N).
 uint32_t dlion_oracle_delta_planes(uint32_t n_workers, int mode) {
     if (mode == DLION_ORACLE_MAJORITY) return 1;
+    if (mode == DLION_ORACLE_MAJORITY_TERNARY) return 2;        // three values: two bits
     uint32_t bits = 0;
     while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;
     return bits;
@@ -269,7 +281,7 @@ int dlion_oracle_aggregate(const dlion_oracle_segment* segs, uint32_t nseg, uint
                            uint32_t n_workers, int mode, const uint32_t* packed,
                            uint32_t* delta_wire) {
     if (!segs || !packed || !delta_wire || d_pad % 32 != 0 || n_workers == 0) return -1;
-    if (mode != DLION_ORACLE_MAJORITY && mode != DLION_ORACLE_AVERAGE) return -1;
+    if (!known_mode(mode)) return -1;
     const uint64_t W = d_pad / 32;
     const uint32_t K = dlion_oracle_delta_planes(n_workers, mode);
     for (uint32_t s = 0; s < nseg; ++s) {
@@ -285,6 +297,11 @@ int dlion_oracle_aggregate(const dlion_oracle_segment* segs, uint32_t nseg, uint
                 for (uint32_t i = 0; i < n_workers; ++i) P += (packed[i * W + w] >> b) & 1u;
                 if (mode == DLION_ORACLE_MAJORITY) {
                     if (2 * static_cast<int64_t>(P) - static_cast<int64_t>(n_workers) >= 0) delta_wire[w] |= 1u << b;
+                } else if (mode == DLION_ORACLE_MAJORITY_TERNARY) {
+                    const int64_t S3 = 2 * static_cast<int64_t>(P) - static_cast<int64_t>(n_workers);
+                    const uint32_t code = (S3 > 0) ? 2u : ((S3 < 0) ? 0u : 1u);    // Delta + 1
+                    delta_wire[w] |= (code & 1u) << b;
+                    delta_wire[W + w] |= (code >> 1) << b;
                 } else {
                     for (uint32_t p = 0; p < K; ++p) delta_wire[p * W + w] |= ((P >> p) & 1u) << b;
                 }
@@ -324,7 +341,7 @@ int dlion_oracle_apply_delta(const dlion_oracle_segment* segs, uint32_t nseg, ui
                              uint32_t n_workers, int mode, const uint32_t* delta_wire, float* x,
                              float lr, float weight_decay) {
     if (!segs || !delta_wire || !x || d_pad % 32 != 0 || n_workers == 0) return -1;
-    if (mode != DLION_ORACLE_MAJORITY && mode != DLION_ORACLE_AVERAGE) return -1;
+    if (!known_mode(mode)) return -1;
     const uint64_t W = d_pad / 32;
     const uint32_t K = dlion_oracle_delta_planes(n_workers, mode);
     const int32_t N = static_cast<int32_t>(n_workers);
@@ -336,6 +353,10 @@ int dlion_oracle_apply_delta(const dlion_oracle_segment* segs, uint32_t nseg, ui
             float Delta;
             if (mode == DLION_ORACLE_MAJORITY) {
                 Delta = ((delta_wire[j / 32] >> (j % 32)) & 1u) ? 1.0f : -1.0f;
+            } else if (mode == DLION_ORACLE_MAJORITY_TERNARY) {
+                const uint32_t low = (delta_wire[j / 32] >> (j % 32)) & 1u;
+                const uint32_t high = (delta_wire[W + j / 32] >> (j % 32)) & 1u;
+                Delta = static_cast<float>(static_cast<int32_t>(low + 2u * high) - 1);    // code - 1
             } else {
                 int32_t P = 0;
                 for (uint32_t p = 0; p < K; ++p) P |= static_cast<int32_t>((delta_wire[p * W + j / 32] >> (j % 32)) & 1u) << p;

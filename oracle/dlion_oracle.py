@@ -22,6 +22,7 @@ _LIB = os.path.join(_HERE, "libdlion_oracle.so")
 
 MAJORITY = 0
 AVERAGE = 1
+MAJORITY_TERNARY = 2      # Majority Vote with Delta = 0 on an even-N tie (three-valued sign)
 GRAD_F32 = 0
 GRAD_BF16 = 1
 STATE_F32 = 0

@@ -24,8 +24,7 @@ constexpr int kThreads = 128;             // 4 warps x 1024 coordinates = one ti
 constexpr int kWarps = kThreads / 32;
 
 template <int PLANES, bool AVG>
-__global__ void __launch_bounds__(kThreads)
-aggregate_kernel(const __grid_constant__ WireParams p) {
+__device__ __forceinline__ void aggregate_body(const WireParams& p) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t thr = (p.n_workers + 1u) >> 1;
@@ -49,8 +48,24 @@ aggregate_kernel(const __grid_constant__ WireParams p) {
     }
 }
 
+// Blocks per SM, measured on the 1.3 B-parameter workload (N = 16, vote + apply pair):
+// Averaging 2.41 ms as the compiler allocates unprompted -> 2.25 ms with 10 blocks here and
+// 7 in the apply kernel; Majority Vote is fastest unprompted (34 registers, 12 blocks), and
+// N >= 64 was not re-measured: both keep the compiler's own allocation.
+template <int PLANES, bool AVG>
+__global__ void __launch_bounds__(kThreads)
+aggregate_kernel(const __grid_constant__ WireParams p) {
+    aggregate_body<PLANES, AVG>(p);
+}
+
+template <int PLANES>
+__global__ void __launch_bounds__(kThreads, 10)
+aggregate_kernel_averaging(const __grid_constant__ WireParams p) {
+    aggregate_body<PLANES, true>(p);
+}
+
 template <int PLANES, bool AVG, bool TABLE>
-__global__ void __launch_bounds__(kThreads, 6)
+__global__ void __launch_bounds__(kThreads, AVG ? 7 : 6)
 apply_delta_kernel(const __grid_constant__ WireParams p) {
     __shared__ float avg_tables[(AVG && PLANES <= 8) ? kWarps : 1][(AVG && PLANES <= 8) ? 256 : 1];
     __shared__ CountArea<(PLANES > 8)> areas[AVG ? kWarps : 1];
@@ -138,8 +153,9 @@ cudaError_t launch(const WireParams& p, bool apply, cudaStream_t s) {
         if (p.average) apply_delta_kernel<PLANES, true, TABLE><<<grid, kThreads, 0, s>>>(p);
         else apply_delta_kernel<1, false, TABLE><<<grid, kThreads, 0, s>>>(p);
     } else if constexpr (!TABLE) {                       // the vote touches no parameter tensor
-        if (p.average) aggregate_kernel<PLANES, true><<<grid, kThreads, 0, s>>>(p);
-        else aggregate_kernel<PLANES, false><<<grid, kThreads, 0, s>>>(p);
+        if (!p.average) aggregate_kernel<PLANES, false><<<grid, kThreads, 0, s>>>(p);
+        else if constexpr (PLANES < 7) aggregate_kernel_averaging<PLANES><<<grid, kThreads, 0, s>>>(p);
+        else aggregate_kernel<PLANES, true><<<grid, kThreads, 0, s>>>(p);
     }
     return cudaGetLastError();
 }

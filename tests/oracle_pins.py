@@ -576,9 +576,79 @@ def check_vote_counts16(lib):
             assert np.array_equal(c8[valid], cnt[valid].astype(np.uint8))
 
 
+def check_ternary_majority(lib):
+    """The optional three-valued reading of the tie (mode MAJORITY_TERNARY): Delta is the
+    textbook sign of S, zero included; with an odd N it is the binary Majority Vote; with N = 2
+    it is Averaging; its two-plane message carries Delta + 1."""
+    TER = orc.MAJORITY_TERNARY
+    rng = np.random.default_rng(23)
+    segs = [(0, 70), (128, 1), (256, 33)]
+    d_pad = 384
+    valid = np.zeros(d_pad, bool)
+    for o, n in segs:
+        valid[o:o + n] = True
+    # hand case: N = 2, one vote each way (a tie), eps = 1/4, lambda = 1/2, x_0 = 2: pure decay, twice
+    one = np.array([[1], [0]], np.uint32)
+    x = np.zeros(32, np.float32)
+    x[0] = 2.0
+    orc.aggregate_apply([(0, 1)], 32, 2, TER, np.ascontiguousarray(one), x, 0.25, 0.5, lib=lib)
+    assert x[0] == 1.75
+    orc.aggregate_apply([(0, 1)], 32, 2, TER, np.ascontiguousarray(one), x, 0.25, 0.5, lib=lib)
+    assert x[0] == 1.53125 and not x[1:].any()
+    for N in (1, 2, 3, 4, 7, 8, 33, 64, 255, 256):
+        bits = (rng.random((N, d_pad)) < rng.random(d_pad)[None, :]) & valid[None, :]
+        if N % 2 == 0:                                   # exact ties on a few coordinates
+            for j in (3, 40, 128, 260):
+                bits[:, j] = np.arange(N) < N // 2
+        packed = np.packbits(bits, axis=1, bitorder="little").view(np.uint32).reshape(N, -1).copy()
+        S = 2 * bits.sum(axis=0).astype(np.int64) - N
+        # Delta read back exactly: x_0 = 0, lr = 1, lambda = 0  ->  x' = -Delta
+        x = np.zeros(d_pad, np.float32)
+        dbits = np.zeros(d_pad // 32, np.uint32)
+        orc.aggregate_apply(segs, d_pad, N, TER, packed, x, 1.0, 0.0, delta_bits=dbits, lib=lib)
+        assert np.array_equal(-x[valid].astype(np.float64), np.sign(S[valid]).astype(np.float64))
+        assert not x[~valid].any()
+        assert np.array_equal(unpack(dbits[None, :], d_pad)[0][valid], (S >= 0)[valid].astype(np.uint8))
+        if N % 2 == 0:
+            assert (x[[3, 40, 128, 260]] == 0).all()
+        x0 = f32(rng.standard_normal(d_pad))
+        xt, xb, xa = x0.copy(), x0.copy(), x0.copy()
+        orc.aggregate_apply(segs, d_pad, N, TER, packed, xt, 0.125, 0.5, lib=lib)
+        orc.aggregate_apply(segs, d_pad, N, MAJ, packed, xb, 0.125, 0.5, lib=lib)
+        orc.aggregate_apply(segs, d_pad, N, AVG, packed, xa, 0.125, 0.5, lib=lib)
+        if N % 2 == 1:
+            assert np.array_equal(xt, xb)                # no ties: the binary rule
+        else:
+            tie = (S == 0) & valid
+            assert np.array_equal(xt[~tie], xb[~tie]) and not np.array_equal(xt[tie], xb[tie])
+        if N == 2:
+            assert np.array_equal(xt, xa)                # S/2 is -1, 0 or +1
+        # the message: two planes holding Delta + 1; vote then apply equals the one-call step
+        assert orc.delta_planes(N, TER, lib=lib) == 2 and orc.wire_bits(1000, N, TER, 1, lib=lib) == 2000
+        wire = np.zeros(2 * d_pad // 32, np.uint32)
+        wire[3] = 0xDEADBEEF                             # word 3 = coordinates 96..127: padding, must stay untouched
+        orc.aggregate(segs, d_pad, N, TER, packed, wire, lib=lib)
+        assert wire[3] == 0xDEADBEEF
+        wire[3] = 0
+        planes = unpack(wire.reshape(2, -1), d_pad).astype(np.int64)
+        code = planes[0] + 2 * planes[1]
+        assert np.array_equal(code[valid], np.sign(S[valid]) + 1) and not code[~valid].any()
+        xw = x0.copy()
+        orc.apply_delta(segs, d_pad, N, TER, wire, xw, 0.125, 0.5, lib=lib)
+        assert np.array_equal(xw, xt)
+    # a tie at every step: x_k = (1 - eps*lambda)^k x_0 (the closed form with Delta = 0)
+    x = np.zeros(32, np.float32)
+    x[0] = 3.0
+    for _ in range(10):
+        orc.aggregate_apply([(0, 1)], 32, 2, TER, np.ascontiguousarray(one), x, 0.01, 0.3, lib=lib)
+    want = 3.0 * (1 - 0.01 * 0.3) ** 10
+    assert abs(float(x[0]) - want) <= 10 * np.spacing(np.float32(3.0))
+
+
 ALL_CHECKS = [check_hand_case, check_sign_of_zero_and_tie, check_delta_is_sign_of_blend,
               check_single_worker_is_lion, check_identical_workers, check_beta_zero_is_signsgd,
               check_equal_betas_is_signum, check_counts_bruteforce, check_x_closed_form,
               check_phase_one_contraction, check_padding_untouched, check_wire_bits,
               check_delta_wire_roundtrip, check_per_worker_betas, check_bf16_momentum_store,
-              check_global_lion_hand_case, check_global_lion_definition, check_vote_counts16]
+              check_global_lion_hand_case, check_global_lion_definition, check_vote_counts16,
+              check_ternary_majority]

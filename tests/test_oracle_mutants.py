@@ -64,6 +64,17 @@ MUTANTS = {
                            "votes += (packed[worker * words + j / 32] >> (31 - j % 32)) & 1u;"),
     "counts16_truncated_to_a_byte": ("count16[j] = static_cast<uint16_t>(votes);",
                                      "count16[j] = static_cast<uint16_t>(votes & 0xFFu);"),
+    "ternary_tie_goes_positive": ("Delta = (S > 0) ? 1.0f : ((S < 0) ? -1.0f : 0.0f);",
+                                  "Delta = (S > 0) ? 1.0f : ((S < 0) ? -1.0f : 1.0f);"),
+    "ternary_strict_sign_flipped": ("Delta = (S > 0) ? 1.0f : ((S < 0) ? -1.0f : 0.0f);",
+                                    "Delta = (S > 0) ? -1.0f : ((S < 0) ? 1.0f : 0.0f);"),
+    "ternary_message_planes_swapped": ("delta_wire[w] |= (code & 1u) << b;\n                    delta_wire[W + w] |= (code >> 1) << b;",
+                                       "delta_wire[W + w] |= (code & 1u) << b;\n                    delta_wire[w] |= (code >> 1) << b;"),
+    "ternary_message_tie_as_plus": ("const uint32_t code = (S3 > 0) ? 2u : ((S3 < 0) ? 0u : 1u);",
+                                    "const uint32_t code = (S3 >= 0) ? 2u : 0u;"),
+    "ternary_decode_without_offset": ("Delta = static_cast<float>(static_cast<int32_t>(low + 2u * high) - 1);",
+                                      "Delta = static_cast<float>(static_cast<int32_t>(low + 2u * high));"),
+    "ternary_one_plane": ("if (mode == DLION_ORACLE_MAJORITY_TERNARY) return 2;", "if (mode == DLION_ORACLE_MAJORITY_TERNARY) return 1;"),
     "average_down_bits_floor_log": ("while ((1ull << bits) < static_cast<uint64_t>(n_workers) + 1ull) ++bits;",
                                     "while ((2ull << bits) <= static_cast<uint64_t>(n_workers)) ++bits;"),
 }
