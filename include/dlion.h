@@ -18,7 +18,8 @@
  *     x' = fl(x - fl(lr*fl(Delta + fl(lambda*x)))); (1-beta) is formed in binary32;
  *     bf16 gradients are widened exactly;
  *   - sign(v) = +1 when v >= 0 (either zero), -1 otherwise (NaN gives -1);
- *   - an even-N tie (S = 0) gives Delta = +1 under Majority Vote;
+ *   - an even-N tie (S = 0) gives Delta = +1 under Majority Vote (Delta = 0 under the
+ *     optional DLION_MAJORITY_TERNARY rule);
  *   - the server's integer is P = number of +1 votes in {0..N}; S = 2P - N;
  *   - Averaging uses the correctly rounded quotient (float)(2P-N) / (float)N.
  *
@@ -68,7 +69,14 @@ typedef enum {
     DLION_ESTATE = 5  /* wrong device current, or context unusable */
 } dlion_status;
 
-typedef enum { DLION_MAJORITY = 0, DLION_AVERAGE = 1 } dlion_mode;
+/* Aggregation rule (Section 3.2).  DLION_MAJORITY_TERNARY is the optional other reading of
+ * an even-N tie: the three-valued sign of the appendix's lemma, sign(0) = 0, so S = 0 gives
+ * Delta = 0 and that coordinate's step is pure weight decay; with an odd N it is
+ * DLION_MAJORITY.  Delta then has three values: the server->worker message is two planes
+ * holding Delta + 1 in {0, 1, 2} (plane 0 = bit 0 = "tie", plane 1 = bit 1 = "S > 0"),
+ * dlion_delta_planes is 2, and dlion_wire_bytes(ctx, 1) counts 2 d bits.  delta_bits_out of
+ * dlion_aggregate_apply stays bit = (S >= 0). */
+typedef enum { DLION_MAJORITY = 0, DLION_AVERAGE = 1, DLION_MAJORITY_TERNARY = 2 } dlion_mode;
 typedef enum { DLION_GRAD_F32 = 0, DLION_GRAD_BF16 = 1 } dlion_gdtype;
 typedef enum { DLION_STATE_F32 = 0, DLION_STATE_BF16 = 1 } dlion_sdtype;
 
@@ -178,7 +186,8 @@ dlion_status dlion_apply_delta_sliced(dlion_ctx* ctx, const uint32_t* delta_wire
                                       float* x, void* cuda_stream);
 
 /* Number of d-bit planes of the server->worker message: 1 for Majority Vote,
- * ceil(log2(N+1)) for Averaging (the paper's "log(N) bits" per parameter).
+ * ceil(log2(N+1)) for Averaging (the paper's "log(N) bits" per parameter), 2 for
+ * DLION_MAJORITY_TERNARY.
  * 0 for a null context. */
 uint32_t dlion_delta_planes(const dlion_ctx* ctx);
 

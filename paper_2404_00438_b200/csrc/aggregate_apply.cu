@@ -66,7 +66,7 @@ __device__ __noinline__ void ragged_tile(const AggParams& p, const TileRef t, ui
         const unsigned long long e = t.base + j0;
         for (uint32_t q = 0; q < 4 && j0 + q < t.valid; ++q) {
             float delta;
-            if constexpr (COUNTS) delta = delta_of_count<PLANES, AVG>(k.c[q], thr, avg_table, p.n_workers);
+            if constexpr (COUNTS) delta = delta_of_count<PLANES, AVG>(k.c[q], thr, avg_table, p.n_workers, p.ternary != 0);
             else delta = ((dn >> q) & 1u) ? 1.0f : -1.0f;
             xs[e + q] = apply_coord(xs[e + q], delta, p.lr, p.wd);
             if constexpr (COUNTS) {
@@ -96,7 +96,7 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
     CountArea<(PLANES > 8)>* area = &areas[COUNTS ? warp : 0];
     bool have_table = !AVG;
     auto fill_table = [&]() {
-        fill_avg_table<PLANES>(avg_table, n, lane);
+        fill_avg_table<PLANES>(avg_table, n, lane, p.ternary != 0);
         have_table = true;
     };
 
@@ -127,10 +127,10 @@ aggregate_apply_kernel(const __grid_constant__ AggParams p) {
             float d0, d1, d2, d3;
             if constexpr (COUNTS) {
                 const Counts4 k = my_counts<PLANES>(area, c, lane);
-                d0 = delta_of_count<PLANES, AVG>(k.c[0], thr, avg_table, n);
-                d1 = delta_of_count<PLANES, AVG>(k.c[1], thr, avg_table, n);
-                d2 = delta_of_count<PLANES, AVG>(k.c[2], thr, avg_table, n);
-                d3 = delta_of_count<PLANES, AVG>(k.c[3], thr, avg_table, n);
+                d0 = delta_of_count<PLANES, AVG>(k.c[0], thr, avg_table, n, p.ternary != 0);
+                d1 = delta_of_count<PLANES, AVG>(k.c[1], thr, avg_table, n, p.ternary != 0);
+                d2 = delta_of_count<PLANES, AVG>(k.c[2], thr, avg_table, n, p.ternary != 0);
+                d3 = delta_of_count<PLANES, AVG>(k.c[3], thr, avg_table, n, p.ternary != 0);
                 if (p.count != nullptr) *reinterpret_cast<uint32_t*>(p.count + xe + c * kChunk) = pack_counts(k);   // N <= 255 here
                 if (p.count16 != nullptr) {
                     *reinterpret_cast<uint2*>(p.count16 + xe + c * kChunk) =

@@ -58,7 +58,9 @@ AggParams agg_params(const dlion_ctx* ctx) {
     p.w_stride = ctx->d_pad / 32;
     p.lr = ctx->lr;
     p.wd = ctx->wd;
-    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    // the three-valued tie rule runs on the Averaging kernels with a table of signs
+    p.ternary = ctx->mode == DLION_MAJORITY_TERNARY ? 1 : 0;
+    p.average = (ctx->mode == DLION_AVERAGE || p.ternary) ? 1 : 0;
     return p;
 }
 
@@ -75,6 +77,7 @@ WireParams wire_params(const dlion_ctx* ctx, uint64_t slice_words) {
     p.lr = ctx->lr;
     p.wd = ctx->wd;
     p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    p.ternary = ctx->mode == DLION_MAJORITY_TERNARY ? 1 : 0;
     return p;
 }
 
@@ -106,7 +109,7 @@ dlion_status dlion_init(dlion_ctx** out, const dlion_segment* segs, uint32_t nse
     if (n_workers == 0 || n_workers > DLION_MAX_WORKERS) return DLION_EINVAL;
     if (!unit_interval(beta1) || !unit_interval(beta2)) return DLION_EINVAL;
     if (!nonneg_finite(lr) || !nonneg_finite(weight_decay)) return DLION_EINVAL;
-    if (mode != DLION_MAJORITY && mode != DLION_AVERAGE) return DLION_EINVAL;
+    if (mode != DLION_MAJORITY && mode != DLION_AVERAGE && mode != DLION_MAJORITY_TERNARY) return DLION_EINVAL;
     if (gdtype != DLION_GRAD_F32 && gdtype != DLION_GRAD_BF16) return DLION_EINVAL;
 
     dlion_ctx* c = new (std::nothrow) dlion_ctx;
@@ -301,7 +304,8 @@ dlion_status dlion_step_fused(dlion_ctx* ctx, const void* grads, void* m, float*
     p.m_bf16 = ctx->sdtype == DLION_STATE_BF16 ? 1 : 0;
     p.lr = ctx->lr;
     p.wd = ctx->wd;
-    p.average = ctx->mode == DLION_AVERAGE ? 1 : 0;
+    p.ternary = ctx->mode == DLION_MAJORITY_TERNARY ? 1 : 0;
+    p.average = (ctx->mode == DLION_AVERAGE || p.ternary) ? 1 : 0;      // ternary: the table variant, with signs in the table
     const cudaError_t e = dlion::launch_step_fused(p, ctx->gdtype == DLION_GRAD_BF16, ctx->sm_count,
                                                    static_cast<cudaStream_t>(cuda_stream));
     if (e != cudaSuccess) return DLION_ECUDA;

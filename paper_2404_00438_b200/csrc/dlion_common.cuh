@@ -233,7 +233,8 @@ struct AggParams {
     unsigned long long ntiles;
     unsigned long long w_stride;     // words between consecutive workers in packed
     float lr, wd;
-    int average;                     // 0 = majority vote, 1 = averaging
+    int average;                     // 0 = majority vote, 1 = averaging (or, with ternary, the same kernel with a sign table)
+    int ternary;                     // Majority Vote with Delta = 0 on an even-N tie
 };
 
 struct FusedParams {
@@ -251,6 +252,7 @@ struct FusedParams {
     int m_bf16;
     float lr, wd;
     int average;
+    int ternary;                     // see AggParams
 };
 
 struct GlobalParams {                // Global-Lion comparison step
@@ -283,6 +285,7 @@ struct WireParams {                  // server-only aggregate / worker-side appl
     unsigned long long slice_words;  // apply: 0, or the message is [slice][plane][slice_words] (all-gather order)
     float lr, wd;
     int average;
+    int ternary;                     // aggregate: write the two planes of Delta + 1 instead of the Delta bit
 };
 
 // One thread block per work item, in item order (the kernels still stride, so a

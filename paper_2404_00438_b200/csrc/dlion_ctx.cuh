@@ -45,5 +45,15 @@ WorkerParams worker_params(const dlion_ctx* c, int worker);
 AggParams agg_params(const dlion_ctx* c);
 WireParams wire_params(const dlion_ctx* c, uint64_t slice_words);
 dlion_status device_ok(const dlion_ctx* c);     // DLION_ESTATE unless the context's device is current
+// The three-valued tie rule's message, Delta + 1 in {0, 1, 2} as two planes, is exactly an
+// Averaging message of a 2-worker problem ((2c - 2) / 2 = c - 1): the apply kernels decode
+// it as such.
+inline void decode_ternary_as_two_workers(WireParams& p) {
+    if (p.ternary) {
+        p.average = 1;
+        p.n_workers = 2;
+        p.kplanes = 2;
+    }
+}
 
 }  // namespace dlion

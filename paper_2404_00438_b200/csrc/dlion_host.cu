@@ -85,7 +85,7 @@ dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, void* m, fl
     // Server side.  The broadcast message, when asked for, is in the format of
     // dlion_aggregate: one plane of Delta bits (Majority Vote) or the K count planes
     // (Averaging; vote and update are then two launches with the message in between).
-    const bool avg = ctx->mode == DLION_AVERAGE;
+    const bool avg = ctx->mode != DLION_MAJORITY;          // more than one plane: vote and apply are two launches
     uint32_t* wire = static_cast<uint32_t*>(delta_wire_dev);
     dlion_status st;
     if (avg && wire != nullptr) {
@@ -106,6 +106,7 @@ dlion_status dlion_step_host(dlion_ctx* ctx, const void* host_grads, void* m, fl
 
 uint32_t dlion_delta_planes(const dlion_ctx* ctx) {
     if (ctx == nullptr) return 0;
+    if (ctx->mode == DLION_MAJORITY_TERNARY) return 2u;       // three values of Delta: two bits
     return ctx->mode == DLION_AVERAGE ? dlion::planes_for(ctx->n_workers) : 1u;
 }
 
@@ -136,6 +137,7 @@ dlion_status dlion_apply_delta_sliced(dlion_ctx* ctx, const uint32_t* delta_wire
     if (cudaGetDevice(&dev) != cudaSuccess) return DLION_ECUDA;
     if (dev != ctx->device) return DLION_ESTATE;
     dlion::WireParams p = dlion::wire_params(ctx, slice_words);
+    dlion::decode_ternary_as_two_workers(p);
     p.wire_in = delta_wire;
     p.x = x;
     if (dlion::launch_wire(p, true, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess) return DLION_ECUDA;
@@ -151,7 +153,9 @@ uint64_t dlion_wire_bytes(const dlion_ctx* ctx, int direction) {
         bits = static_cast<uint64_t>(ctx->n_workers) * d;
     } else if (direction == 1) {
         uint32_t per = 1;
-        if (ctx->mode == DLION_AVERAGE) {
+        if (ctx->mode == DLION_MAJORITY_TERNARY) {
+            per = 2;
+        } else if (ctx->mode == DLION_AVERAGE) {
             per = 0;
             while ((1ull << per) < static_cast<uint64_t>(ctx->n_workers) + 1) ++per;   // N+1 values
         }

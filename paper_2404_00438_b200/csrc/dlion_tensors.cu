@@ -133,6 +133,7 @@ dlion_status dlion_apply_delta_tensors(dlion_ctx* ctx, const uint32_t* delta_wir
     const dlion_status ds = dlion::device_ok(ctx);
     if (ds != DLION_OK) return ds;
     dlion::WireParams p = dlion::wire_params(ctx, slice_words);
+    dlion::decode_ternary_as_two_workers(p);
     p.wire_in = delta_wire;
     p.x = reinterpret_cast<float*>(ctx->tables_dev);
     p.x_off = ctx->tables_dev + 2 * static_cast<size_t>(ctx->n_workers) * ctx->nseg;

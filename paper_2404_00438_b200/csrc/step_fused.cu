@@ -97,8 +97,10 @@ step_fused_kernel(const __grid_constant__ FusedParams p) {
     const uint32_t n = p.n_workers;
     if constexpr (AVG) {
         for (uint32_t c = threadIdx.x; c <= n; c += kThreads) {
-            avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
-                                     static_cast<float>(n));
+            const int sum = 2 * static_cast<int>(c) - static_cast<int>(n);
+            // Averaging's quotient; or, for the three-valued tie rule, the sign of the sum with sign(0) = 0
+            avg_table[c] = p.ternary ? (sum > 0 ? 1.0f : (sum < 0 ? -1.0f : 0.0f))
+                                     : __fdiv_rn(static_cast<float>(sum), static_cast<float>(n));
         }
         __syncthreads();
     }

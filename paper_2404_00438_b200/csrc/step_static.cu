@@ -72,7 +72,7 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
     if (n_workers == 0 || n_workers > DLION_MAX_WORKERS) return DLION_EINVAL;
     if (!unit_interval(beta1) || !unit_interval(beta2)) return DLION_EINVAL;
     if (!nonneg_finite(lr) || !nonneg_finite(weight_decay)) return DLION_EINVAL;
-    if (mode != DLION_MAJORITY && mode != DLION_AVERAGE) return DLION_EINVAL;
+    if (mode != DLION_MAJORITY && mode != DLION_AVERAGE && mode != DLION_MAJORITY_TERNARY) return DLION_EINVAL;
     if (gdtype != DLION_GRAD_F32 && gdtype != DLION_GRAD_BF16) return DLION_EINVAL;
     if (d > kMaxCoordWorkers) return DLION_EINVAL;
     const unsigned long long d_pad = (d + DLION_ALIGN - 1) / DLION_ALIGN * DLION_ALIGN;
@@ -125,7 +125,8 @@ extern "C" dlion_status dlion_step_static(uint64_t d, uint32_t n_workers, float 
     ap.w_stride = d_pad / 32;
     ap.lr = lr;
     ap.wd = weight_decay;
-    ap.average = mode == DLION_AVERAGE ? 1 : 0;
+    ap.ternary = mode == DLION_MAJORITY_TERNARY ? 1 : 0;
+    ap.average = (mode == DLION_AVERAGE || ap.ternary) ? 1 : 0;
     if (dlion::launch_aggregate_apply(ap, pd.sm_count, s) != cudaSuccess) return DLION_ECUDA;
     return DLION_OK;
 }

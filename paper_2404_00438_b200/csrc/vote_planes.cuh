@@ -202,25 +202,35 @@ __device__ __forceinline__ uint32_t my_delta_bits(uint32_t dword, int c, uint32_
     return (__shfl_sync(kFull, dword, 4u * c + (lane >> 3)) >> (4u * (lane & 7u))) & 0xFu;
 }
 
+// Delta as a function of the vote count P where it is tabulated or computed from P:
+// Averaging's correctly rounded quotient (2P - N) / N, or -- the optional three-valued
+// tie rule, which runs on the Averaging kernels with this other table -- the sign of
+// 2P - N with sign(0) = 0.
+__device__ __forceinline__ float delta_value(uint32_t count, uint32_t n, bool ternary) {
+    const int s = 2 * static_cast<int>(count) - static_cast<int>(n);
+    if (ternary) return s > 0 ? 1.0f : (s < 0 ? -1.0f : 0.0f);
+    return __fdiv_rn(static_cast<float>(s), static_cast<float>(n));
+}
+
 // Delta of a coordinate from its vote count P.  Majority Vote: +1 iff P >= ceil(N/2).
-// Averaging: from the per-warp table while the counts fit it (N <= 255), else the
-// correctly rounded quotient directly.
+// Averaging (and the three-valued tie rule): from the per-warp table while the counts fit
+// it (N <= 255), else computed directly.
 template <int PLANES, bool AVG>
-__device__ __forceinline__ float delta_of_count(uint32_t count, uint32_t thr, const float* avg_table, uint32_t n) {
+__device__ __forceinline__ float delta_of_count(uint32_t count, uint32_t thr, const float* avg_table, uint32_t n,
+                                                bool ternary) {
     if constexpr (AVG) {
         if constexpr (PLANES <= 8) return avg_table[count];
-        return __fdiv_rn(static_cast<float>(2 * static_cast<int>(count) - static_cast<int>(n)), static_cast<float>(n));
+        return delta_value(count, n, ternary);
     }
     return count >= thr ? 1.0f : -1.0f;
 }
 
 // Fills a warp's private table of Averaging's Delta for every count (N <= 255 only).
 template <int PLANES>
-__device__ __forceinline__ void fill_avg_table(float* avg_table, uint32_t n, uint32_t lane) {
+__device__ __forceinline__ void fill_avg_table(float* avg_table, uint32_t n, uint32_t lane, bool ternary) {
     if constexpr (PLANES <= 8) {
         for (uint32_t c = lane; c <= n; c += 32) {
-            avg_table[c] = __fdiv_rn(static_cast<float>(2 * static_cast<int>(c) - static_cast<int>(n)),
-                                     static_cast<float>(n));
+            avg_table[c] = delta_value(c, n, ternary);
         }
         __syncwarp();
     }

@@ -23,7 +23,9 @@ namespace {
 constexpr int kThreads = 128;             // 4 warps x 1024 coordinates = one tile
 constexpr int kWarps = kThreads / 32;
 
-template <int PLANES, bool AVG>
+// TERNARY (Majority Vote only): the three-valued tie rule's two-plane message.  A template
+// parameter: as a run-time test it cost the plain Majority-Vote vote 3 %.
+template <int PLANES, bool AVG, bool TERNARY>
 __device__ __forceinline__ void aggregate_body(const WireParams& p) {
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
@@ -42,6 +44,12 @@ __device__ __forceinline__ void aggregate_body(const WireParams& p) {
             for (int q = 0; q < PLANES; ++q) {
                 if (q < static_cast<int>(p.kplanes)) p.wire_out[q * p.plane_stride + word_idx] = pl[q] & vmask;
             }
+        } else if constexpr (TERNARY) {
+            // the three-valued rule: Delta + 1 in {0, 1, 2} as two planes (bit 0 = tie, bit 1 = S > 0)
+            const uint32_t ge = planes_ge<PLANES>(pl, thr);
+            const uint32_t tie = (p.n_workers & 1u) ? 0u : (ge & ~planes_ge<PLANES>(pl, thr + 1u));
+            p.wire_out[word_idx] = tie & vmask;
+            p.wire_out[p.plane_stride + word_idx] = ge & ~tie & vmask;
         } else {
             p.wire_out[word_idx] = planes_ge<PLANES>(pl, thr) & vmask;
         }
@@ -52,16 +60,16 @@ __device__ __forceinline__ void aggregate_body(const WireParams& p) {
 // Averaging 2.41 ms as the compiler allocates unprompted -> 2.25 ms with 10 blocks here and
 // 7 in the apply kernel; Majority Vote is fastest unprompted (34 registers, 12 blocks), and
 // N >= 64 was not re-measured: both keep the compiler's own allocation.
-template <int PLANES, bool AVG>
+template <int PLANES, bool AVG, bool TERNARY>
 __global__ void __launch_bounds__(kThreads)
 aggregate_kernel(const __grid_constant__ WireParams p) {
-    aggregate_body<PLANES, AVG>(p);
+    aggregate_body<PLANES, AVG, TERNARY>(p);
 }
 
 template <int PLANES>
 __global__ void __launch_bounds__(kThreads, 10)
 aggregate_kernel_averaging(const __grid_constant__ WireParams p) {
-    aggregate_body<PLANES, true>(p);
+    aggregate_body<PLANES, true, false>(p);
 }
 
 template <int PLANES, bool AVG, bool TABLE>
@@ -107,7 +115,7 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
                             ? __ldg(p.wire_in + q * p.plane_stride + at) : 0u;
             }
             if (!have_table) {
-                fill_avg_table<PLANES>(avg_table, n, lane);
+                fill_avg_table<PLANES>(avg_table, n, lane, false);
                 have_table = true;
             }
             publish_counts<PLANES>(pl, area, lane);
@@ -120,7 +128,7 @@ apply_delta_kernel(const __grid_constant__ WireParams p) {
             if constexpr (AVG) {
                 const Counts4 k = my_counts<PLANES>(area, c, lane);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) d[q] = delta_of_count<PLANES, true>(k.c[q], 0u, avg_table, n);
+                for (int q = 0; q < 4; ++q) d[q] = delta_of_count<PLANES, true>(k.c[q], 0u, avg_table, n, false);
             } else {
                 const uint32_t dn = my_delta_bits(dword, c, lane);
 #pragma unroll
@@ -153,9 +161,10 @@ cudaError_t launch(const WireParams& p, bool apply, cudaStream_t s) {
         if (p.average) apply_delta_kernel<PLANES, true, TABLE><<<grid, kThreads, 0, s>>>(p);
         else apply_delta_kernel<1, false, TABLE><<<grid, kThreads, 0, s>>>(p);
     } else if constexpr (!TABLE) {                       // the vote touches no parameter tensor
-        if (!p.average) aggregate_kernel<PLANES, false><<<grid, kThreads, 0, s>>>(p);
+        if (p.ternary) aggregate_kernel<PLANES, false, true><<<grid, kThreads, 0, s>>>(p);
+        else if (!p.average) aggregate_kernel<PLANES, false, false><<<grid, kThreads, 0, s>>>(p);
         else if constexpr (PLANES < 7) aggregate_kernel_averaging<PLANES><<<grid, kThreads, 0, s>>>(p);
-        else aggregate_kernel<PLANES, true><<<grid, kThreads, 0, s>>>(p);
+        else aggregate_kernel<PLANES, true, false><<<grid, kThreads, 0, s>>>(p);
     }
     return cudaGetLastError();
 }

@@ -15,7 +15,7 @@ import torch
 
 from . import build as _build
 
-MAJORITY, AVERAGE = 0, 1
+MAJORITY, AVERAGE, MAJORITY_TERNARY = 0, 1, 2
 GRAD_F32, GRAD_BF16 = 0, 1
 STATE_F32, STATE_BF16 = 0, 1
 ALIGN = 128

@@ -29,6 +29,7 @@ import torch
 ALIGN = 128            # segment starts are multiples of this many elements
 MAJORITY = 0
 AVERAGE = 1
+MAJORITY_TERNARY = 2      # Majority Vote with Delta = 0 on an even-N tie
 _MASK64 = (1 << 64) - 1
 _TABLE_BITS = 16
 _CHUNK = 1 << 24       # elements generated per pass (bounds temporaries)

@@ -51,7 +51,7 @@ def test_check_layout(dl):
 
 @pytest.mark.parametrize("kw", [
     dict(n_workers=0), dict(n_workers=65536), dict(beta1=-0.1), dict(beta1=1.5), dict(beta2=float("nan")),
-    dict(lr=-1.0), dict(lr=float("inf")), dict(weight_decay=-0.5), dict(mode=2), dict(gdtype=7),
+    dict(lr=-1.0), dict(lr=float("inf")), dict(weight_decay=-0.5), dict(mode=3), dict(gdtype=7),
 ])
 def test_init_rejects_bad_arguments_before_cuda(dl, kw):
     args = dict(n_workers=4, beta1=0.9, beta2=0.99, lr=1e-4, weight_decay=0.1, mode=0, gdtype=0)
