@@ -390,6 +390,7 @@ def run_ours(args):
             barrier()
             return statistics.mean(e[t].elapsed_time(e[t + 1]) for t in range(args.steps))
 
+        time.sleep(1.0)        # these stages are timed alone: let the power state of the timed region settle
         extra["other_rule_ms"] = timed(lambda: ctx2.aggregate_apply(packed, x_scratch))
         extra["other_rule"] = "average" if other else "majority"
         if args.state == "f32":
