@@ -373,20 +373,37 @@ def run_full(dl, w: inputs.Workload, steps: int, path: str = "two_stage",
 
 def cross_check_paths(dl, w: inputs.Workload, steps: int, mode: int) -> None:
     """Whole arenas, no CPU work: the product paths that promise identical bits -- the
-    two-stage step, per-worker calls followed by dlion_aggregate + dlion_apply_delta, and the
-    one-launch step -- are run side by side on the same gradients and must leave identical
-    momentum, parameters and sign words everywhere, padding included.  (The oracle anchors the
-    two-stage path; this extends that anchor to every coordinate of the other paths.)"""
+    two-stage step; per-worker calls followed by dlion_aggregate + dlion_apply_delta; the
+    one-launch step; the per-tensor mode (every tensor bound as its own pointer); and the
+    scatter mode (sign words stored into four per-slice receive buffers, then voted on slice
+    by slice and applied from the gathered message) -- are run side by side on the same
+    gradients and must leave identical momentum, parameters and sign words everywhere,
+    padding included.  (The oracle anchors the two-stage path; this extends that anchor to
+    every coordinate of the other paths.)"""
     dev = torch.device("cuda:0")
     N, D, W = w.n_workers, w.d_pad, w.d_pad // 32
     gdt = inputs.grad_torch_dtype(w)
     ctx = make_ctx(dl, w, mode)
     g = torch.empty(N, D, dtype=gdt, device=dev)
     x0 = inputs.fill_x0(w, torch.empty(D, device=dev))
-    ms = [torch.zeros(N, D, device=dev) for _ in range(3)]
-    xs = [x0.clone() for _ in range(3)]
-    ps = [torch.zeros(N, W, dtype=torch.int32, device=dev) for _ in range(3)]
-    wire = torch.zeros(ctx.delta_planes() * W, dtype=torch.int32, device=dev)
+    P = 5
+    ms = [torch.zeros(N, D, device=dev) for _ in range(P)]
+    xs = [x0.clone() for _ in range(P)]
+    ps = [torch.zeros(N, W, dtype=torch.int32, device=dev) for _ in range(4)]
+    K = ctx.delta_planes()
+    wire = torch.zeros(K * W, dtype=torch.int32, device=dev)
+    # per-tensor mode: its own context; every tensor is a view into arenas 3
+    tctx = make_ctx(dl, w, mode)
+    tctx.bind_tensors(grads=[[g[i, o:o + k] for o, k in w.segments] for i in range(N)],
+                      m=[[ms[3][i, o:o + k] for o, k in w.segments] for i in range(N)],
+                      x=[xs[3][o:o + k] for o, k in w.segments])
+    # scatter mode: four slices when the arena splits evenly, else two or one
+    S = next(k for k in (4, 2, 1) if W % (4 * k) == 0)     # every slice a whole number of 128-coordinate groups
+    SW = W // S
+    sctx = make_ctx(dl, w, mode)
+    server = dl.Dlion([(0, D // S)], D // S, N, w.beta1, w.beta2, w.lr, w.weight_decay, mode, gdtype_of(w))
+    recv = [torch.zeros(N, SW, dtype=torch.int32, device=dev) for _ in range(S)]
+    gathered = torch.zeros(S, K, SW, dtype=torch.int32, device=dev)
     for t in range(steps):
         inputs.fill_grads(w, t, g)
         ctx.worker_step(-1, g, ms[0], ps[0])
@@ -396,9 +413,22 @@ def cross_check_paths(dl, w: inputs.Workload, steps: int, mode: int) -> None:
         ctx.aggregate(ps[1], wire)
         ctx.apply_delta(wire, xs[1])
         ctx.step_fused(g, ms[2], xs[2], ps[2])
+        tctx.worker_step_tensors(-1, ps[3])
+        tctx.aggregate_apply_tensors(ps[3])
+        for i in range(N):
+            sctx.bind_scatter(recv, SW, slot=i, rows=N)
+            sctx.worker_step_scatter(i, g[i], ms[4][i])
+        for q in range(S):
+            server.aggregate(recv[q], gathered[q])
+        ctx.apply_delta_sliced(gathered, SW, xs[4])
         torch.cuda.synchronize()
-        for k, name in ((1, "per-worker + wire"), (2, "fused")):
-            assert torch.equal(ms[k], ms[0]), f"{w.name} step {t}: momentum of the {name} path differs"
-            assert torch.equal(xs[k], xs[0]), f"{w.name} step {t}: parameters of the {name} path differ"
-            assert torch.equal(ps[k], ps[0]), f"{w.name} step {t}: sign words of the {name} path differ"
-    ctx.destroy()
+        names = ("two-stage", "per-worker + wire", "fused", "per-tensor", "scatter")
+        for k in range(1, P):
+            assert torch.equal(ms[k], ms[0]), f"{w.name} step {t}: momentum of the {names[k]} path differs"
+            assert torch.equal(xs[k], xs[0]), f"{w.name} step {t}: parameters of the {names[k]} path differ"
+        for k in range(1, 4):
+            assert torch.equal(ps[k], ps[0]), f"{w.name} step {t}: sign words of the {names[k]} path differ"
+        for q in range(S):
+            assert torch.equal(recv[q], ps[0][:, q * SW:(q + 1) * SW]), f"{w.name} step {t}: receive buffer {q} differs"
+    for c in (ctx, tctx, sctx, server):
+        c.destroy()

@@ -38,6 +38,8 @@ def test_c2_gpt2_small_table(dl):
     _free()
     assert gp.run_full(dl, w, 3, "fused", modes=(AVG,)) == 0
     _free()
+    assert gp.run_full(dl, w, 5, modes=(AVG,), state="bf16") == 0        # bf16 momentum: every coordinate too
+    _free()
     gp.cross_check_paths(dl, w, 3, AVG)
     _free()
 
