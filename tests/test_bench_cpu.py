@@ -35,3 +35,16 @@ def test_algorithmic_bytes():
     assert bench.bytes_per_param_k2(w) == 10.0
     assert bench.bytes_per_param_worker_k1(inputs.workload("c1")) == 12.125
     assert bench.host_memory_available() > 0
+
+
+def test_traffic_record_matches_the_committed_kernel_sources():
+    """profiles/ncu_traffic.json is keyed by a hash of the worker-side kernel's sources: the
+    record in the tree must be the one captured from the sources in the tree, and close to the
+    algorithmic bytes (a capture with wasted re-reads would show here)."""
+    sys.path.insert(0, ROOT)
+    import bench
+    f32 = bench.ncu_traffic("worker_step_kernel", "grads_bf16_momentum_f32")
+    b16 = bench.ncu_traffic("worker_step_kernel", "grads_bf16_momentum_bf16")
+    assert f32 is not None and b16 is not None, "kernel sources changed since the ncu capture: capture again"
+    assert 0.97 * 10.125 <= f32 <= 1.03 * 10.125 and 0.97 * 6.125 <= b16 <= 1.03 * 6.125
+    assert bench.ncu_traffic("worker_step_kernel", "no_such_variant") is None

@@ -84,7 +84,7 @@ def _worker(rank, world, port, mode, out_dir):
         dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("world,mode", [(2, 0), (2, 1), (3, 0), (4, 1)])
+@pytest.mark.parametrize("world,mode", [(2, 0), (2, 1), (3, 0), (4, 1), (2, 2), (4, 2)])
 def test_exchange_equals_single_process_step(world, mode, tmp_path, oracle):
     mp.spawn(_worker, args=(world, _free_port(), mode, str(tmp_path)), nprocs=world, join=True)
     assert all((tmp_path / f"ok{r}").exists() for r in range(world))

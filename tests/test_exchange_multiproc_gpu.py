@@ -60,7 +60,7 @@ def _rank(rank, world, port, mode, gd, out_dir):
         dist.destroy_process_group()
 
 
-@pytest.mark.parametrize("world,mode,gd", [(2, 0, "f32"), (2, 1, "bf16"), (3, 1, "f32"), (4, 0, "bf16"), (4, 1, "f32")])
+@pytest.mark.parametrize("world,mode,gd", [(2, 0, "f32"), (2, 1, "bf16"), (3, 1, "f32"), (4, 0, "bf16"), (4, 1, "f32"), (2, 2, "f32")])
 def test_processes_sharing_one_gpu_equal_the_oracle(world, mode, gd, tmp_path):
     assert torch.cuda.is_available()
     from paper_2404_00438_b200 import build
