@@ -439,6 +439,11 @@ def run_ours(args):
             exch = run_exchange(args, w, mode, dev, world, rank, barrier)
         except Exception as e:                        # reported, never allowed to take the main line down
             exch = {"error": f"{type(e).__name__}: {e}"}
+        if args.exchange_fused_send and "error" not in exch:
+            try:
+                exch["fused_send"] = run_exchange(args, w, mode, dev, world, rank, barrier, fused_send=True)
+            except Exception as e:
+                exch["fused_send"] = {"error": f"{type(e).__name__}: {e}"}
 
     # ---- end to end: gradients in pinned host memory, Delta read back
     e2e = None
@@ -616,7 +621,7 @@ def run_server_stage(args):
     ctx.destroy()
 
 
-def run_exchange(args, w, mode, dev, world, rank, barrier):
+def run_exchange(args, w, mode, dev, world, rank, barrier, fused_send=False):
     """The paper's own deployment, one worker per GPU: worker-side kernel on this rank's
     gradients, all-to-all of the 1-bit shards, vote on this rank's coordinate slice,
     all-gather of the broadcast message, apply (exchange.DistributedLion; the collectives
@@ -634,7 +639,7 @@ def run_exchange(args, w, mode, dev, world, rank, barrier):
     try:
         opt = exchange.DistributedLion(w.segments, w.d_pad, mode, beta1=w.beta1, beta2=w.beta2, lr=w.lr,
                                        weight_decay=w.weight_decay, gdtype=0 if w.grad_dtype == "f32" else 1,
-                                       device=dev)
+                                       device=dev, fused_send=fused_send)
         Dx = opt.d_pad_x
         g = torch.zeros(Dx, dtype=inputs.grad_torch_dtype(w), device=dev)
         inputs.fill_grads(w, 0, g[:w.d_pad].unsqueeze(0), workers=[rank % max(w.n_workers, 1)])
@@ -657,7 +662,10 @@ def run_exchange(args, w, mode, dev, world, rank, barrier):
         ms = float(t.item()) / args.steps
         sent, received = opt.wire_bytes_per_step()
         return {"ms_per_step": ms, "value": w.d * world / (ms * 1e-3) / 1e9, "unit": UNIT, "workers": world,
-                "steps": args.steps, "gpu_launches_per_step": 3, "collectives": "all_to_all_single + all_gather_into_tensor (NCCL)",
+                "steps": args.steps, "gpu_launches_per_step": 3,
+                "collectives": ("sign words stored by the worker-side kernel into the ranks' receive buffers "
+                                "(symmetric memory) + barrier + all_gather_into_tensor (NCCL)") if fused_send
+                else "all_to_all_single + all_gather_into_tensor (NCCL)",
                 "alltoall_bytes_sent_per_rank": sent, "allgather_bytes_received_per_rank": received,
                 "fp32_ring_allreduce_bytes_per_rank": int(2 * (world - 1) / world * 4 * w.d),
                 "note": "one worker per GPU, d = the workload's parameter count on every rank"}
@@ -714,6 +722,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--exchange", action="store_true",
                     help="also time the worker = GPU exchange step (always on with more than one rank)")
+    ap.add_argument("--exchange-fused-send", action="store_true",
+                    help="with the exchange leg: time it once more with the all-to-all fused into the worker-side "
+                         "kernel (peer stores into symmetric memory); only on request")
     ap.add_argument("--no-extra", action="store_true",
                     help="skip the stages timed after the timed region (other aggregation rule, Global Lion)")
     ap.add_argument("--e2e-steps", type=int, default=2)
