@@ -168,8 +168,11 @@ def bytes_per_param_k2(w) -> float:
     return w.n_workers / 8 + 4 + 4
 
 
+MODE_NAMES = {inputs.MAJORITY: "majority", inputs.AVERAGE: "average", inputs.MAJORITY_TERNARY: "ternary"}
+
+
 def mode_of(name: str) -> int:
-    return {"majority": inputs.MAJORITY, "average": inputs.AVERAGE}[name]
+    return {v: k for k, v in MODE_NAMES.items()}[name]
 
 
 def oracle_sample_rate(w, mode: int, seconds: float, nthreads: int, n_max: int = 1 << 22):
@@ -231,7 +234,7 @@ def run_reference(args):
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
         "data": "synthetic",
         "config": {"workload": args.workload, "n_workers": w.n_workers, "d": w.d,
-                   "mode": "average" if mode else "majority", "grads": w.grad_dtype},
+                   "mode": MODE_NAMES[mode], "grads": w.grad_dtype},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": "each step: " + sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -393,7 +396,7 @@ def run_ours(args):
 
         time.sleep(1.0)        # these stages are timed alone: let the power state of the timed region settle
         extra["other_rule_ms"] = timed(lambda: ctx2.aggregate_apply(packed, x_scratch))
-        extra["other_rule"] = "average" if other else "majority"
+        extra["other_rule"] = MODE_NAMES[other]
         if N <= 255:                                   # the one-launch step counts votes in bytes
             extra["fused_ms"] = timed(lambda: ctx.step_fused(g, m, x_scratch, None))
         if args.state == "f32":
@@ -476,7 +479,7 @@ def run_ours(args):
             b2 = w.d * bytes_per_param_k2(w)
             if args.path == "wire":                   # votes in, K planes out; K planes in, x in and out
                 b2 += 2 * w.d * ctx.delta_planes() / 8
-            rule = "average" if mode else "majority"
+            rule = MODE_NAMES[mode]
             key = ("aggregate_kernel+apply_delta_kernel<%s>" if args.path == "wire" else "aggregate_apply_kernel<%s>") % rule
             stages = {key: {"achieved": b2 / (k2 * 1e-3) / 1e9, "unit": "GB/s",
                             "frac": b2 / (k2 * 1e-3) / 1e9 / peak,
@@ -494,7 +497,7 @@ def run_ours(args):
             if "fused_ms" in extra:
                 bf = w.d * (N * (w.grad_bytes + 2 * sbytes) + 8)
                 msf = extra["fused_ms"]
-                stages["step_fused_kernel<%s>" % ("average" if mode else "majority")] = {
+                stages["step_fused_kernel<%s>" % MODE_NAMES[mode]] = {
                     "achieved": bf / (msf * 1e-3) / 1e9, "unit": "GB/s", "frac": bf / (msf * 1e-3) / 1e9 / peak,
                     "frac_of_8tbs_nominal": bf / (msf * 1e-3) / 1e9 / 8000.0, "ms_per_launch": msf,
                     "algorithmic_bytes_per_launch": bf,
@@ -525,7 +528,7 @@ def run_ours(args):
             "warmup": args.warmup, "ms_per_step": total_ms_max / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": args.workload, "n_workers": N, "d": w.d, "grads": w.grad_dtype,
-                       "mode": "average" if mode else "majority", "path": args.path,
+                       "mode": MODE_NAMES[mode], "path": args.path,
                        "momentum": args.state,
                        "l2": "inputs larger than L2 (no flush needed)" if N * D * (w.grad_bytes + 4) > 4 * 126e6
                              else "working set comparable to L2: latency-bound case",
@@ -609,7 +612,7 @@ def run_server_stage(args):
         "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": k2,
         "ms_min": min(ms), "higher_is_better": True, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "n_workers": N, "d": w.d, "stage": "server",
-                   "mode": "average" if mode else "majority",
+                   "mode": MODE_NAMES[mode],
                    "l2": "votes + x = %.0f MB, larger than L2" % ((N * D / 8 + 4 * D) / 1e6)},
         "roofline": {"bound": "hbm", "kernel": "aggregate_apply_kernel", "achieved": achieved, "peak": 8000.0,
                      "unit": "GB/s", "frac": achieved / 8000.0, "peak_source": "nominal 8 TB/s",
@@ -712,7 +715,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5"])
     ap.add_argument("--n-workers", type=int, default=0, help="override N (the c4 sweep)")
-    ap.add_argument("--mode", default=None, choices=["majority", "average"])
+    ap.add_argument("--mode", default=None, choices=["majority", "average", "ternary"],
+                    help="ternary: Majority Vote with Delta = 0 on an even-N tie")
     ap.add_argument("--path", default="two_stage", choices=["two_stage", "fused", "wire"],
                     help="wire: server side as two launches with the broadcast message in between")
     ap.add_argument("--state", default="f32", choices=["f32", "bf16"], help="momentum storage")
