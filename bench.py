@@ -539,6 +539,10 @@ def run_ours(args):
             "exchange": exch, "cpu_baseline": cpu, "e2e": e2e,
             "gpu_launches": launches, "clocks": clocks,
             "wire_bytes_per_step": {"up_all_workers": up, "down_per_worker": down,
+                                    # Averaging: the paper's own estimate, log2(N) bits per parameter (the exact
+                                    # count of N+1 values is ceil(log2(N+1)), which `down_per_worker` uses)
+                                    "down_per_worker_paper_log2_n": (w.d * np.log2(N) / 8 if mode == inputs.AVERAGE and N > 1
+                                                                     else None),
                                     "fp32_gradients_each_way_per_worker": ctx.wire_bytes(2),
                                     "fp32_ring_allreduce_per_gpu": int(2 * (N - 1) / N * 4 * w.d)},
         }
