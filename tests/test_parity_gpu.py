@@ -584,3 +584,45 @@ def test_calls_can_be_captured_in_a_cuda_graph(dl):
         a, b = run(True, fused), run(False, fused)
         assert all(torch.equal(u, v) for u, v in zip(a, b))
     ctx.destroy()
+
+
+def test_checkpoint_and_resume_is_bit_identical(dl):
+    """The library keeps no optimizer state of its own: saving m and x to the host after two
+    steps, destroying the context, and resuming in a new context from the saved copies gives the
+    same bits as four uninterrupted steps (per-worker betas and bf16 momentum included)."""
+    dev = torch.device("cuda:0")
+    n = 5
+    w = inputs.custom(RAGGED, n, AVG, "bf16", scale=1e-3, lr=1e-3, weight_decay=0.5)
+    D, W = w.d_pad, w.d_pad // 32
+
+    def new_ctx():
+        c = gp.make_ctx(dl, w)
+        c.set_momentum_dtype(dl.STATE_BF16)
+        c.set_worker_betas(3, 0.5, 0.5)
+        return c
+
+    grads = [inputs.fill_grads(w, t, torch.empty(n, D, dtype=torch.bfloat16)).to(dev) for t in range(4)]
+    x0 = inputs.fill_x0(w, torch.empty(D))
+    packed = torch.zeros(n, W, dtype=torch.int32, device=dev)
+    ctx = new_ctx()
+    m_a, x_a = torch.zeros(n, D, dtype=torch.bfloat16, device=dev), x0.to(dev)
+    for t in range(4):
+        ctx.worker_step(-1, grads[t], m_a, packed)
+        ctx.aggregate_apply(packed, x_a)
+    ctx.destroy()
+    ctx = new_ctx()
+    m_b, x_b = torch.zeros(n, D, dtype=torch.bfloat16, device=dev), x0.to(dev)
+    for t in range(2):
+        ctx.worker_step(-1, grads[t], m_b, packed)
+        ctx.aggregate_apply(packed, x_b)
+    torch.cuda.synchronize()
+    saved_m, saved_x = m_b.cpu().clone(), x_b.cpu().clone()            # the checkpoint
+    ctx.destroy()
+    del m_b, x_b
+    ctx = new_ctx()
+    m_c, x_c = saved_m.to(dev), saved_x.to(dev)
+    for t in range(2, 4):
+        ctx.step_fused(grads[t], m_c, x_c, None)                       # resumed on another path, too
+    torch.cuda.synchronize()
+    assert torch.equal(m_c.view(torch.int16), m_a.view(torch.int16)) and torch.equal(x_c, x_a)
+    ctx.destroy()
