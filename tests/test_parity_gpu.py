@@ -323,6 +323,24 @@ def test_random_configurations(dl, seed):
         assert gp.run_small(dl, w, 3, path, modes=(mode,)) == 0
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_random_configurations_three_valued_tie_rule(dl, seed):
+    """The same kind of random configuration under the three-valued tie rule; even worker counts
+    are favoured so that ties occur."""
+    rng = np.random.default_rng(5000 + seed)
+    numels = [int(rng.choice([0, 1, 33, 129, 4096, 4097, int(rng.integers(1, 20000)), int(rng.integers(1, 3 * 4096 * 4))]))
+              for _ in range(int(rng.integers(1, 7)))]
+    n = int(rng.choice([1, 2, 2, 4, 4, 6, 8, 9, 16, 32, 64, 100, 254, 255]))
+    gd = str(rng.choice(["f32", "bf16"]))
+    w = inputs.custom(numels, n, inputs.MAJORITY_TERNARY, gd, scale=1.0 if gd == "f32" else 1e-3,
+                      a_private=float(rng.choice([0.5, 1.0, 2.0])), beta1=float(rng.choice([0.0, 0.9, 0.95])),
+                      beta2=float(rng.choice([0.0, 0.99, 0.999])), lr=float(rng.choice([1e-4, 1e-2, 0.25])),
+                      weight_decay=float(rng.choice([0.0, 0.1, 1.0])), zero_frac=float(rng.choice([0.0, 0.05])),
+                      seed=int(rng.integers(0, 1 << 30)))
+    for path in ("two_stage", "fused"):
+        assert gp.run_small(dl, w, 3, path, modes=(inputs.MAJORITY_TERNARY,)) == 0
+
+
 # ---------------------------------------------------------------- guard bands
 @pytest.mark.parametrize("gd,state", [("f32", "f32"), ("bf16", "f32"), ("bf16", "bf16")])
 def test_nothing_is_written_outside_the_arenas(dl, gd, state):
