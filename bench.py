@@ -667,8 +667,34 @@ def run_exchange(args, w, mode, dev, world, rank, barrier, fused_send=False):
         if world > 1:
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item()) / args.steps
+        phases = None
+        if not fused_send:
+            # the same step once more, phase by phase (events on the launching stream; the
+            # collectives are enqueued on it by the backend): where a multi-GPU step spends its time
+            names = ("worker_step", "all_to_all", "vote_on_slice", "all_gather", "apply")
+            acc = [0.0] * len(names)
+            for _ in range(args.steps):
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)]
+                ev[0].record(stream)
+                opt.kernels.worker_step(g, m, opt.packed)
+                ev[1].record(stream)
+                opt._all_to_all()
+                ev[2].record(stream)
+                opt.kernels.aggregate(opt.recv, opt.wire_slice)
+                ev[3].record(stream)
+                opt._all_gather()
+                ev[4].record(stream)
+                opt.kernels.apply_delta_sliced(opt.gathered, opt.slice_words, x)
+                ev[5].record(stream)
+                torch.cuda.synchronize()
+                for k in range(len(names)):
+                    acc[k] += ev[k].elapsed_time(ev[k + 1])
+            pt = torch.tensor(acc, dtype=torch.float64, device=dev) / args.steps
+            if world > 1:
+                dist.all_reduce(pt, op=dist.ReduceOp.MAX)
+            phases = {nm: float(v) for nm, v in zip(names, pt.tolist())}
         sent, received = opt.wire_bytes_per_step()
-        return {"ms_per_step": ms, "value": w.d * world / (ms * 1e-3) / 1e9, "unit": UNIT, "workers": world,
+        return {"ms_per_step": ms, "phases_ms_max_over_ranks": phases, "value": w.d * world / (ms * 1e-3) / 1e9, "unit": UNIT, "workers": world,
                 "steps": args.steps, "gpu_launches_per_step": 3,
                 "collectives": ("sign words stored by the worker-side kernel into the ranks' receive buffers "
                                 "(symmetric memory) + barrier + all_gather_into_tensor (NCCL)") if fused_send
