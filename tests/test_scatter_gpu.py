@@ -39,7 +39,12 @@ def test_scattered_signs_complete_the_exchange(dl, world, mode, gd, state):
     if state == "bf16":
         model.set_momentum_dtype(dl.STATE_BF16)
     K = model.delta_planes()
-    recv = [torch.zeros(world, SW, dtype=torch.int32, device=dev) for _ in range(world)]     # rank q's receive buffer
+    # rank q's receive buffer, each inside its own allocation between two bands of a sentinel value
+    GUARD, SENTINEL = 256, 0x5A5A5A5A
+    backing = [torch.full((world * SW + 2 * GUARD,), SENTINEL, dtype=torch.int32, device=dev) for _ in range(world)]
+    recv = [b[GUARD:GUARD + world * SW].view(world, SW) for b in backing]
+    for r_ in recv:
+        r_.zero_()
     gathered = torch.zeros(world, K, SW, dtype=torch.int32, device=dev)
     x0 = torch.zeros(D)
     x0[:w.d_pad] = inputs.fill_x0(w, torch.empty(w.d_pad))
@@ -69,6 +74,8 @@ def test_scattered_signs_complete_the_exchange(dl, world, mode, gd, state):
         got_m = got_m.numpy() if state == "f32" else got_m.view(torch.int16).numpy().view(np.uint16)
         gp.compare(f"step {t} m", got_m, m_ref, True)
         gp.compare(f"step {t} x", x.cpu().numpy(), x_ref, True)
+    for b in backing:                                   # nothing was stored outside a receive buffer
+        assert bool((b[:GUARD] == SENTINEL).all()) and bool((b[GUARD + world * SW:] == SENTINEL).all())
     # argument checks
     with pytest.raises(dl.DlionError) as e:
         model.bind_scatter(recv[:-1], SW, 0, world)                    # slices do not cover the arena
