@@ -473,7 +473,10 @@ def run_ours(args):
         roofline = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_source": peak_src, "frac_of_8tbs_nominal": achieved / 8000.0,
                     "algorithmic_bytes_per_launch": alg_bytes, "ms_per_launch": k1,
-                    "traffic": None if traffic is None else traffic * w.d * N}
+                    "traffic": None if traffic is None else traffic * w.d * N,
+                    # duration x median SM clock of the timed region: compares runs taken at different
+                    # power-cap clocks (a DRAM-bound kernel's product rises with the clock, an issue-bound one's does not)
+                    "ms_per_launch_x_sm_ghz": (k1 * clocks["sm_mhz"] / 1000.0 if clocks and clocks.get("sm_mhz") else None)}
         stages = None
         if args.path != "fused":
             b2 = w.d * bytes_per_param_k2(w)
